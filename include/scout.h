@@ -1,0 +1,206 @@
+/*
+ * scout.h - C ABI of the B200 (sm_100a) sign+vote library.
+ *
+ * The data-parallel hot path of Consensus Collective Communication (C3):
+ * a compact signature for every chunk of R equivalent replicas' tensors, then
+ * strict-majority voting over the signatures to name the outlier replicas and
+ * the chunks they corrupt.  R replicas are R sets of buffers in one GPU's
+ * memory.
+ *
+ * Conventions
+ *   - plain C; every function returns int: SCOUT_OK (0) or a negative error;
+ *     nothing throws, aborts or takes ownership of caller memory;
+ *   - "device" pointers are CUDA device addresses valid on the current device,
+ *     "host" pointers are ordinary host memory;
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream);
+ *     work is enqueued there and, except for scout_certify, the call returns
+ *     without waiting for it;
+ *   - the library allocates device memory only inside a plan object;
+ *   - the replica index is the position in the caller's pointer table: this is
+ *     the ordered peer-to-rank map that C3 stores with its result (Sec. 5.1).
+ */
+#ifndef SCOUT_H
+#define SCOUT_H
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define SCOUT_API __attribute__((visibility("default")))
+#else
+#define SCOUT_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    SCOUT_OK = 0,
+    SCOUT_ERR_INVALID = -1,     /* bad argument (NULL, R out of range, size 0, ...)     */
+    SCOUT_ERR_ALIGN = -2,       /* a tensor address is not 16-byte aligned              */
+    SCOUT_ERR_UNSUPPORTED = -3, /* valid request this build does not implement (R > 64) */
+    SCOUT_ERR_CUDA = -4,        /* a CUDA runtime call failed; see scout_last_cuda_error */
+    SCOUT_ERR_NOMEM = -5,       /* host or device allocation failed                     */
+    SCOUT_ERR_TRUNCATED = -6    /* a result list was shorter than needed; counters hold
+                                   the true totals, entries beyond capacity were dropped */
+};
+
+/* Element types.  The code enters the signature (the evidence covers the dtype,
+ * Sec. 5.2), so the numbering is frozen. */
+enum {
+    SCOUT_DT_U8 = 0, SCOUT_DT_F32 = 1, SCOUT_DT_BF16 = 2, SCOUT_DT_I64 = 3,
+    SCOUT_DT_F16 = 4, SCOUT_DT_F64 = 5, SCOUT_DT_I32 = 6
+};
+
+/* The three statuses of a C3 result (Sec. 5.1): they keep an all-zero bitmap
+ * from being ambiguous. */
+enum { SCOUT_AGREE = 0, SCOUT_ATTRIBUTED = 1, SCOUT_INCONCLUSIVE = 2 };
+
+/* Verdict of scout_certify over a whole replicated state. */
+enum { SCOUT_CERTIFIED = 0, SCOUT_VERDICT_ATTRIBUTED = 1, SCOUT_UNDECIDED = 2 };
+
+typedef struct scout_plan scout_plan_t; /* opaque; owns its device tables and scratch */
+
+/* Comparable evidence of one (chunk, replica) (Sec. 5.2).  Only `hash` is
+ * compared by the vote; the other fields are a diagnostic sidecar. */
+typedef struct {
+    uint64_t hash;      /* 64-bit position-sensitive signature of dtype, shape tag, bytes */
+    uint32_t nan_count; /* elements that are NaN (0 for integer types)                   */
+    uint32_t inf_count; /* elements that are +-Inf                                       */
+    double sum;         /* sum of the finite elements                                    */
+    double sumsq;       /* sum of squares of the finite elements                         */
+} scout_sig_t;          /* 32 bytes */
+
+typedef struct {
+    uint64_t nbytes;   /* > 0, a multiple of the element size                  */
+    uint32_t dtype;    /* SCOUT_DT_*                                            */
+    uint32_t reserved; /* must be 0                                             */
+    uint64_t meta_tag; /* caller's shape tag (scout_shape_tag), 0 allowed       */
+} scout_tensor_t;
+
+typedef struct {
+    uint64_t chunk;    /* global chunk id                                       */
+    uint32_t replica;  /* index of the outlier replica                          */
+    uint32_t reserved;
+} scout_outlier_t;     /* 16 bytes */
+
+typedef struct {
+    uint64_t n_chunks, n_agree, n_attributed, n_inconclusive;
+    uint64_t n_outliers, n_undecided; /* true totals even if a list was truncated   */
+    uint64_t replica_union_bitmap;    /* OR of every chunk's outlier bitmap          */
+    uint64_t certificate;             /* digest of the majority hashes; 0 if UNDECIDED */
+    int32_t verdict;                  /* SCOUT_CERTIFIED / _VERDICT_ATTRIBUTED / _UNDECIDED */
+    int32_t reserved;
+} scout_report_t;
+
+/* ---- plan: chunking ------------------------------------------------------
+ * Cuts every tensor into pieces of `chunk_bytes` (the last piece short; pieces
+ * never span tensors).  The global chunk id runs over (tensor, piece).  The
+ * chunk is this library's unit of evidence: C3 is applied once per chunk, so a
+ * disagreement is localised to (replica, chunk) instead of (replica, tensor)
+ * as in Sec. 5.2.
+ *   R            number of replicas, 2..64 (a singleton has no comparison,
+ *                Sec. 4 "Peer-group size"; more than 64 needs a wider bitmap:
+ *                SCOUT_ERR_UNSUPPORTED)
+ *   T, tensors   host array of T descriptors, copied
+ *   chunk_bytes  a multiple of 512, at most 1 GiB
+ *   out          receives the plan; destroy with scout_plan_destroy
+ * Allocates the device tables and the per-tile scratch on the current device. */
+SCOUT_API int scout_plan_create(uint32_t R, uint64_t T, const scout_tensor_t *tensors /*host*/,
+                      uint64_t chunk_bytes, scout_plan_t **out);
+
+/* ptrs: host array of R*T device addresses, replica-major (ptrs[r*T + t] is
+ * tensor t of replica r), each 16-byte aligned (else SCOUT_ERR_ALIGN) and
+ * readable for tensors[t].nbytes.  The table is copied to the device on the
+ * default stream; the buffers stay the caller's.  May be called again to scan
+ * other buffers of the same geometry. */
+SCOUT_API int scout_plan_bind(scout_plan_t *plan, const void *const *ptrs /*host*/);
+
+SCOUT_API int scout_plan_num_chunks(const scout_plan_t *plan, uint64_t *C);
+SCOUT_API int scout_plan_chunk_info(const scout_plan_t *plan, uint64_t c, uint64_t *tensor,
+                          uint64_t *index_in_tensor, uint64_t *byte_offset, uint64_t *nbytes);
+SCOUT_API int scout_plan_destroy(scout_plan_t *plan);
+
+/* ---- comparable evidence (Sec. 5.2: e_i = H_w(dtype, shape, bytes)) -------
+ * Reads every byte of every bound replica once and writes one record per
+ * (chunk, replica) to d_sigs[c*R + r] (device, C*R records).  The bulk fold and
+ * the finalisation both run on the device (Sec. 9 folds on the device and
+ * finalises on the host; here only the records leave the kernel).
+ * Asynchronous on `stream`.  Results are bitwise reproducible for a given plan. */
+SCOUT_API int scout_sign_chunks(scout_plan_t *plan, void *stream, scout_sig_t *d_sigs /*device [C][R]*/);
+
+/* ---- exact consensus (Sec. 5.3; Algorithm 1, Exact branch) ----------------
+ * Per chunk: the most frequent hash e* and its count c*.  If c* <= R/2 the
+ * chunk is SCOUT_INCONCLUSIVE with bitmap 0 and its id is appended to
+ * d_undecided; otherwise bit j of the bitmap is 1{e_j != e*}, the status is
+ * SCOUT_ATTRIBUTED if any bit is set, else SCOUT_AGREE, and (chunk, j) is
+ * appended to d_outliers for every set bit.
+ *   d_sigs                   device [C][R] records (only .hash is compared)
+ *   d_status, d_bitmap       device [C]; either may be NULL
+ *   d_outliers, d_undecided  device lists of the given capacities (NULL with
+ *                            capacity 0 allowed); entries are in no particular
+ *                            order; entries beyond capacity are dropped
+ *   d_counts                 device [6]: n_chunks, n_agree, n_attributed,
+ *                            n_inconclusive, n_outliers, n_undecided (true totals)
+ * Asynchronous on `stream`; overflow of a list is visible as count > capacity. */
+SCOUT_API int scout_consensus_vote(uint32_t R, uint64_t C, const scout_sig_t *d_sigs, uint8_t *d_status,
+                         uint64_t *d_bitmap, scout_outlier_t *d_outliers, uint64_t outlier_cap,
+                         uint64_t *d_undecided, uint64_t undecided_cap, uint64_t *d_counts,
+                         void *stream);
+
+/* ---- certify a replicated state -------------------------------------------
+ * sign + vote + roll-up over everything bound to the plan (the optimizer-
+ * boundary comparison of Sec. 9 extended from a sampled slice to the full
+ * state; a checkpoint is worth promoting only if its replicas agree, Sec. 8).
+ * Synchronises `stream`.  Host lists come back sorted by (chunk, replica).
+ * Returns SCOUT_ERR_TRUNCATED (report still valid) if a list was too short.
+ *   verdict CERTIFIED   every chunk agrees
+ *           ATTRIBUTED  every chunk has a strict majority; replica_union_bitmap
+ *                       names the bad replicas, the others are certified
+ *           UNDECIDED   at least one chunk has no strict majority; no certificate */
+SCOUT_API int scout_certify(scout_plan_t *plan, void *stream, scout_report_t *report /*host*/,
+                  scout_outlier_t *h_outliers /*host*/, uint64_t outlier_cap,
+                  uint64_t *h_undecided /*host*/, uint64_t undecided_cap);
+
+/* After scout_certify: device pointers to the plan-owned results of that run
+ * (valid until the next certify or destroy).  Any output may be NULL. */
+SCOUT_API int scout_plan_results(const scout_plan_t *plan, const scout_sig_t **d_sigs,
+                       const uint8_t **d_status, const uint64_t **d_bitmap);
+/* After scout_certify: chunks attributed to each replica, host [R]. */
+SCOUT_API int scout_plan_replica_bad_counts(const scout_plan_t *plan, uint64_t *h_counts /*host [R]*/);
+
+/* Tensor-level signatures, the granularity of Sec. 5.2: for every (tensor,
+ * replica) the chunk hashes folded in order.  d_sigs: device [C][R] records;
+ * d_tensor_sigs: device [T][R].  Asynchronous on `stream`. */
+SCOUT_API int scout_rollup_tensors(const scout_plan_t *plan, const scout_sig_t *d_sigs,
+                         uint64_t *d_tensor_sigs /*device [T][R]*/, void *stream);
+
+/* Same as scout_certify for replicas that live in HOST memory (checkpoints kept
+ * in CPU memory, Sec. 8): h_ptrs is a host array of R*T host addresses,
+ * replica-major.  The data is streamed through plan-owned device staging
+ * buffers in slices, copy overlapped with signing.  Pinned host memory copies
+ * faster; pageable memory works.  Synchronous. */
+SCOUT_API int scout_certify_host(scout_plan_t *plan, const void *const *h_ptrs /*host*/,
+                       scout_report_t *report /*host*/, scout_outlier_t *h_outliers,
+                       uint64_t outlier_cap, uint64_t *h_undecided, uint64_t undecided_cap);
+
+/* Shape tag for scout_tensor_t.meta_tag: a 64-bit digest of (ndim, dims). */
+SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/);
+
+/* Tuning knobs of a plan (optional; call before the first scout_sign_chunks).
+ * key "tile_bytes": bytes per work item, a power of two in [2048, 65536];
+ * key "variant": 0 = direct vector loads, 1 = bulk-async staging through
+ * shared memory.  Results do not depend on either except for the rounding
+ * order of the floating-point sums. */
+SCOUT_API int scout_plan_set(scout_plan_t *plan, const char *key, int64_t value);
+SCOUT_API int scout_plan_get(const scout_plan_t *plan, const char *key, int64_t *value);
+
+SCOUT_API const char *scout_strerror(int code);
+SCOUT_API int scout_version(void);
+/* Name of the CUDA error behind the calling thread's most recent SCOUT_ERR_CUDA ("" if none). */
+SCOUT_API const char *scout_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SCOUT_H */

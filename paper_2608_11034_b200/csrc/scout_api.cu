@@ -1,0 +1,535 @@
+// Host side of the C ABI: plan construction (chunk and tile tables), argument
+// validation, launch sequencing, and the certify roll-up.  All arithmetic of the
+// method runs in the kernels of scout_sign.cu and scout_vote.cu.
+#include <algorithm>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "scout_internal.h"
+
+namespace scout {
+
+static thread_local std::string g_last_cuda_error;
+
+void set_cuda_error(cudaError_t e, const char *what) {
+    g_last_cuda_error = std::string(cudaGetErrorName(e)) + ": " + cudaGetErrorString(e) + " in " + what;
+    (void)cudaGetLastError();  // clear the sticky-free error state
+}
+
+static uint32_t dtype_size(uint32_t d) {
+    switch (d) {
+        case SCOUT_DT_U8: return 1;
+        case SCOUT_DT_F32: return 4;
+        case SCOUT_DT_BF16: return 2;
+        case SCOUT_DT_I64: return 8;
+        case SCOUT_DT_F16: return 2;
+        case SCOUT_DT_F64: return 8;
+        case SCOUT_DT_I32: return 4;
+        default: return 0;
+    }
+}
+
+}  // namespace scout
+
+using namespace scout;
+
+struct scout_plan {
+    uint32_t R = 0;
+    uint64_t T = 0, chunk_bytes = 0;
+    std::vector<scout_tensor_t> tensors;
+    std::vector<ChunkDesc> chunks;
+    std::vector<uint64_t> tensor_chunk0;  // [T+1]
+    std::vector<uint64_t> tensor_poff;    // [T+1] packed offsets, 256-byte aligned
+    std::vector<TileDesc> tiles;
+    uint32_t tile_bytes = 0;
+    int variant = 0, device = 0, grid = 0;
+    bool bound = false;
+
+    TileDesc *d_tiles = nullptr;
+    ChunkDesc *d_chunks = nullptr;
+    uint64_t *d_tensor_chunk0 = nullptr;
+    const uint8_t **d_ptrs = nullptr;
+    TileRec *d_recs = nullptr;
+
+    // certify-owned results
+    scout_sig_t *d_sigs = nullptr;
+    uint8_t *d_status = nullptr;
+    uint64_t *d_bitmap = nullptr, *d_majority = nullptr, *d_undecided = nullptr;
+    scout_outlier_t *d_outliers = nullptr;
+    uint64_t outlier_cap = 0, undecided_cap = 0;
+    CertifyOut *d_out = nullptr, *h_out = nullptr;
+    bool have_results = false;
+
+    // host-replica staging
+    uint8_t *d_stage[2] = {nullptr, nullptr};
+    uint64_t stage_bytes = 0;
+    cudaStream_t s_copy = nullptr, s_comp = nullptr;
+    cudaEvent_t ev_copied[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr};
+};
+
+namespace {
+
+uint32_t auto_tile_bytes(uint64_t total_bytes) {
+    // aim for several work items per resident warp; 2 KiB .. 32 KiB, power of two
+    const uint64_t want_items = 148ull * 32 * 8;
+    uint64_t t = total_bytes / want_items;
+    uint32_t tile = 2048;
+    while (tile < 32768 && (uint64_t)tile * 2 <= t) tile *= 2;
+    return tile;
+}
+
+void build_tiles(scout_plan *p) {
+    p->tiles.clear();
+    for (uint64_t c = 0; c < p->chunks.size(); ++c) {
+        ChunkDesc &cd = p->chunks[c];
+        cd.tile0 = p->tiles.size();
+        uint32_t n = 0;
+        for (uint64_t o = 0; o < cd.nbytes; o += p->tile_bytes, ++n) {
+            TileDesc td;
+            td.off = cd.byte_offset + o;
+            td.poff = p->tensor_poff[cd.tensor] + td.off;
+            td.tensor = cd.tensor;
+            td.nbytes = (uint32_t)std::min<uint64_t>(p->tile_bytes, cd.nbytes - o);
+            td.chunk = (uint32_t)c;
+            td.dtype = cd.dtype;
+            p->tiles.push_back(td);
+        }
+        cd.ntiles = n;
+    }
+}
+
+int upload_tables(scout_plan *p) {
+    if (p->d_tiles) { cudaFree(p->d_tiles); p->d_tiles = nullptr; }
+    if (p->d_recs) { cudaFree(p->d_recs); p->d_recs = nullptr; }
+    if (p->d_chunks) { cudaFree(p->d_chunks); p->d_chunks = nullptr; }
+    const size_t nt = p->tiles.size(), nc = p->chunks.size();
+    SCOUT_CUDA(cudaMalloc(&p->d_tiles, nt * sizeof(TileDesc)));
+    SCOUT_CUDA(cudaMalloc(&p->d_chunks, nc * sizeof(ChunkDesc)));
+    SCOUT_CUDA(cudaMalloc(&p->d_recs, nt * p->R * sizeof(TileRec)));
+    SCOUT_CUDA(cudaMemcpy(p->d_tiles, p->tiles.data(), nt * sizeof(TileDesc), cudaMemcpyHostToDevice));
+    SCOUT_CUDA(cudaMemcpy(p->d_chunks, p->chunks.data(), nc * sizeof(ChunkDesc), cudaMemcpyHostToDevice));
+    return SCOUT_OK;
+}
+
+int sign_all(scout_plan *p, cudaStream_t stream, scout_sig_t *d_sigs) {
+    SignLaunch l;
+    l.tiles = p->d_tiles;
+    l.tile_begin = 0;
+    l.n_tiles = p->tiles.size();
+    l.tiles_per_replica = p->tiles.size();
+    l.replica_begin = 0;
+    l.n_replicas = p->R;
+    l.ptrs = (const uint8_t *const *)p->d_ptrs;
+    l.T = p->T;
+    l.stage = nullptr;
+    l.slice_begin = 0;
+    l.recs = p->d_recs;
+    l.variant = p->variant;
+    l.grid = p->grid;
+    int rc = launch_sign_tiles(l, stream);
+    if (rc) return rc;
+    return launch_finalize(p->d_chunks, p->chunks.size(), p->R, p->d_recs, p->tiles.size(),
+                           p->tile_bytes / ROW_BYTES, d_sigs, stream);
+}
+
+int ensure_certify_buffers(scout_plan *p, uint64_t outlier_cap, uint64_t undecided_cap) {
+    const uint64_t C = p->chunks.size();
+    if (!p->d_sigs) {
+        SCOUT_CUDA(cudaMalloc(&p->d_sigs, C * p->R * sizeof(scout_sig_t)));
+        SCOUT_CUDA(cudaMalloc(&p->d_status, C));
+        SCOUT_CUDA(cudaMalloc(&p->d_bitmap, C * sizeof(uint64_t)));
+        SCOUT_CUDA(cudaMalloc(&p->d_majority, C * sizeof(uint64_t)));
+        SCOUT_CUDA(cudaMalloc(&p->d_out, sizeof(CertifyOut)));
+        SCOUT_CUDA(cudaMallocHost(&p->h_out, sizeof(CertifyOut)));
+    }
+    if (!p->d_outliers || outlier_cap > p->outlier_cap) {
+        if (p->d_outliers) cudaFree(p->d_outliers);
+        p->d_outliers = nullptr;
+        p->outlier_cap = std::max<uint64_t>(outlier_cap, 1);
+        SCOUT_CUDA(cudaMalloc(&p->d_outliers, p->outlier_cap * sizeof(scout_outlier_t)));
+    }
+    if (!p->d_undecided || undecided_cap > p->undecided_cap) {
+        if (p->d_undecided) cudaFree(p->d_undecided);
+        p->d_undecided = nullptr;
+        p->undecided_cap = std::max<uint64_t>(undecided_cap, 1);
+        SCOUT_CUDA(cudaMalloc(&p->d_undecided, p->undecided_cap * sizeof(uint64_t)));
+    }
+    return SCOUT_OK;
+}
+
+// vote + certificate + copy-back + host canonicalisation, after d_sigs is ready on `stream`
+int vote_and_report(scout_plan *p, cudaStream_t stream, scout_report_t *report,
+                    scout_outlier_t *h_outliers, uint64_t outlier_cap, uint64_t *h_undecided,
+                    uint64_t undecided_cap) {
+    const uint64_t C = p->chunks.size();
+    int rc = launch_vote(p->R, C, p->d_sigs, p->d_status, p->d_bitmap, p->d_outliers, outlier_cap,
+                         p->d_undecided, undecided_cap, p->d_out->counts, p->d_majority, p->d_out,
+                         stream);
+    if (rc) return rc;
+    rc = launch_certificate(C, p->d_majority, p->d_out, stream);
+    if (rc) return rc;
+    SCOUT_CUDA(cudaMemcpyAsync(p->h_out, p->d_out, sizeof(CertifyOut), cudaMemcpyDeviceToHost, stream));
+    SCOUT_CUDA(cudaStreamSynchronize(stream));
+    const CertifyOut &o = *p->h_out;
+    const uint64_t n_out = std::min<uint64_t>(o.counts[4], outlier_cap);
+    const uint64_t n_und = std::min<uint64_t>(o.counts[5], undecided_cap);
+    if (n_out)
+        SCOUT_CUDA(cudaMemcpyAsync(h_outliers, p->d_outliers, n_out * sizeof(scout_outlier_t),
+                                   cudaMemcpyDeviceToHost, stream));
+    if (n_und)
+        SCOUT_CUDA(cudaMemcpyAsync(h_undecided, p->d_undecided, n_und * sizeof(uint64_t),
+                                   cudaMemcpyDeviceToHost, stream));
+    if (n_out || n_und) SCOUT_CUDA(cudaStreamSynchronize(stream));
+    // device lists are in arrival order; the host lists are canonical
+    std::sort(h_outliers, h_outliers + n_out, [](const scout_outlier_t &a, const scout_outlier_t &b) {
+        return a.chunk != b.chunk ? a.chunk < b.chunk : a.replica < b.replica;
+    });
+    std::sort(h_undecided, h_undecided + n_und);
+    std::memset(report, 0, sizeof(*report));
+    report->n_chunks = o.counts[0];
+    report->n_agree = o.counts[1];
+    report->n_attributed = o.counts[2];
+    report->n_inconclusive = o.counts[3];
+    report->n_outliers = o.counts[4];
+    report->n_undecided = o.counts[5];
+    report->replica_union_bitmap = o.union_bitmap;
+    report->certificate = o.certificate;
+    report->verdict = o.counts[3] ? SCOUT_UNDECIDED
+                                  : (o.counts[2] ? SCOUT_VERDICT_ATTRIBUTED : SCOUT_CERTIFIED);
+    p->have_results = true;
+    return (o.counts[4] > outlier_cap || o.counts[5] > undecided_cap) ? SCOUT_ERR_TRUNCATED : SCOUT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int scout_plan_create(uint32_t R, uint64_t T, const scout_tensor_t *tensors, uint64_t chunk_bytes,
+                      scout_plan_t **out) {
+    if (!out) return SCOUT_ERR_INVALID;
+    *out = nullptr;
+    if (R < 2 || !tensors || T == 0) return SCOUT_ERR_INVALID;
+    if (R > 64) return SCOUT_ERR_UNSUPPORTED;
+    if (chunk_bytes == 0 || chunk_bytes % ROW_BYTES != 0 || chunk_bytes > (1ull << 30))
+        return SCOUT_ERR_INVALID;
+    if (T > 0xFFFFFFFFull) return SCOUT_ERR_UNSUPPORTED;
+    scout_plan *p = new (std::nothrow) scout_plan;
+    if (!p) return SCOUT_ERR_NOMEM;
+    p->R = R;
+    p->T = T;
+    p->chunk_bytes = chunk_bytes;
+    uint64_t total = 0, poff = 0;
+    try {
+        p->tensors.assign(tensors, tensors + T);
+        p->tensor_chunk0.resize(T + 1);
+        p->tensor_poff.resize(T + 1);
+        for (uint64_t t = 0; t < T; ++t) {
+            const scout_tensor_t &tn = tensors[t];
+            const uint32_t es = dtype_size(tn.dtype);
+            if (es == 0 || tn.nbytes == 0 || tn.nbytes % es != 0 || tn.reserved != 0) {
+                delete p;
+                return SCOUT_ERR_INVALID;
+            }
+            p->tensor_chunk0[t] = p->chunks.size();
+            p->tensor_poff[t] = poff;
+            poff += (tn.nbytes + 255) / 256 * 256;
+            total += tn.nbytes;
+            uint64_t k = 0;
+            for (uint64_t o = 0; o < tn.nbytes; o += chunk_bytes, ++k) {
+                ChunkDesc cd;
+                std::memset(&cd, 0, sizeof(cd));
+                cd.nbytes = std::min<uint64_t>(chunk_bytes, tn.nbytes - o);
+                cd.k = k;
+                cd.meta = tn.meta_tag;
+                cd.dtype = tn.dtype;
+                cd.tensor = (uint32_t)t;
+                cd.byte_offset = o;
+                p->chunks.push_back(cd);
+            }
+        }
+        p->tensor_chunk0[T] = p->chunks.size();
+        p->tensor_poff[T] = poff;
+        if (p->chunks.size() > 0xFFFFFFFFull) {
+            delete p;
+            return SCOUT_ERR_UNSUPPORTED;
+        }
+        p->tile_bytes = auto_tile_bytes(total * R);
+        build_tiles(p);
+    } catch (const std::bad_alloc &) {
+        delete p;
+        return SCOUT_ERR_NOMEM;
+    }
+    int rc = SCOUT_OK;
+    do {
+        if (cudaGetDevice(&p->device) != cudaSuccess) { rc = SCOUT_ERR_CUDA; break; }
+        if ((rc = sign_grid_size(p->variant, p->device, &p->grid))) break;
+        if ((rc = upload_tables(p))) break;
+        if (cudaMalloc(&p->d_tensor_chunk0, (T + 1) * sizeof(uint64_t)) != cudaSuccess ||
+            cudaMalloc(&p->d_ptrs, (size_t)R * T * sizeof(void *)) != cudaSuccess) {
+            rc = SCOUT_ERR_NOMEM;
+            break;
+        }
+        if (cudaMemcpy(p->d_tensor_chunk0, p->tensor_chunk0.data(), (T + 1) * sizeof(uint64_t),
+                       cudaMemcpyHostToDevice) != cudaSuccess) {
+            rc = SCOUT_ERR_CUDA;
+            break;
+        }
+    } while (0);
+    if (rc) {
+        scout_plan_destroy(p);
+        return rc;
+    }
+    *out = p;
+    return SCOUT_OK;
+}
+
+int scout_plan_bind(scout_plan_t *p, const void *const *ptrs) {
+    if (!p || !ptrs) return SCOUT_ERR_INVALID;
+    const uint64_t n = (uint64_t)p->R * p->T;
+    for (uint64_t i = 0; i < n; ++i) {
+        if (!ptrs[i]) return SCOUT_ERR_INVALID;
+        if ((uintptr_t)ptrs[i] & 15u) return SCOUT_ERR_ALIGN;
+    }
+    SCOUT_CUDA(cudaMemcpy(p->d_ptrs, ptrs, n * sizeof(void *), cudaMemcpyHostToDevice));
+    p->bound = true;
+    return SCOUT_OK;
+}
+
+int scout_plan_num_chunks(const scout_plan_t *p, uint64_t *C) {
+    if (!p || !C) return SCOUT_ERR_INVALID;
+    *C = p->chunks.size();
+    return SCOUT_OK;
+}
+
+int scout_plan_chunk_info(const scout_plan_t *p, uint64_t c, uint64_t *tensor, uint64_t *index_in_tensor,
+                          uint64_t *byte_offset, uint64_t *nbytes) {
+    if (!p || c >= p->chunks.size()) return SCOUT_ERR_INVALID;
+    const ChunkDesc &cd = p->chunks[c];
+    if (tensor) *tensor = cd.tensor;
+    if (index_in_tensor) *index_in_tensor = cd.k;
+    if (byte_offset) *byte_offset = cd.byte_offset;
+    if (nbytes) *nbytes = cd.nbytes;
+    return SCOUT_OK;
+}
+
+int scout_plan_destroy(scout_plan_t *p) {
+    if (!p) return SCOUT_OK;
+    cudaFree(p->d_tiles);
+    cudaFree(p->d_chunks);
+    cudaFree(p->d_tensor_chunk0);
+    cudaFree((void *)p->d_ptrs);
+    cudaFree(p->d_recs);
+    cudaFree(p->d_sigs);
+    cudaFree(p->d_status);
+    cudaFree(p->d_bitmap);
+    cudaFree(p->d_majority);
+    cudaFree(p->d_undecided);
+    cudaFree(p->d_outliers);
+    cudaFree(p->d_out);
+    if (p->h_out) cudaFreeHost(p->h_out);
+    for (int i = 0; i < 2; ++i) {
+        cudaFree(p->d_stage[i]);
+        if (p->ev_copied[i]) cudaEventDestroy(p->ev_copied[i]);
+        if (p->ev_done[i]) cudaEventDestroy(p->ev_done[i]);
+    }
+    if (p->s_copy) cudaStreamDestroy(p->s_copy);
+    if (p->s_comp) cudaStreamDestroy(p->s_comp);
+    (void)cudaGetLastError();
+    delete p;
+    return SCOUT_OK;
+}
+
+int scout_sign_chunks(scout_plan_t *p, void *stream, scout_sig_t *d_sigs) {
+    if (!p || !d_sigs) return SCOUT_ERR_INVALID;
+    if (!p->bound) return SCOUT_ERR_INVALID;
+    return sign_all(p, (cudaStream_t)stream, d_sigs);
+}
+
+int scout_consensus_vote(uint32_t R, uint64_t C, const scout_sig_t *d_sigs, uint8_t *d_status,
+                         uint64_t *d_bitmap, scout_outlier_t *d_outliers, uint64_t outlier_cap,
+                         uint64_t *d_undecided, uint64_t undecided_cap, uint64_t *d_counts,
+                         void *stream) {
+    if (R < 2) return SCOUT_ERR_INVALID;
+    if (R > 64) return SCOUT_ERR_UNSUPPORTED;
+    if (!d_counts || (C && !d_sigs)) return SCOUT_ERR_INVALID;
+    if ((outlier_cap && !d_outliers) || (undecided_cap && !d_undecided)) return SCOUT_ERR_INVALID;
+    return launch_vote(R, C, d_sigs, d_status, d_bitmap, d_outliers, outlier_cap, d_undecided,
+                       undecided_cap, d_counts, nullptr, nullptr, (cudaStream_t)stream);
+}
+
+int scout_certify(scout_plan_t *p, void *stream, scout_report_t *report, scout_outlier_t *h_outliers,
+                  uint64_t outlier_cap, uint64_t *h_undecided, uint64_t undecided_cap) {
+    if (!p || !report || !p->bound) return SCOUT_ERR_INVALID;
+    if ((outlier_cap && !h_outliers) || (undecided_cap && !h_undecided)) return SCOUT_ERR_INVALID;
+    int rc = ensure_certify_buffers(p, outlier_cap, undecided_cap);
+    if (rc) return rc;
+    cudaStream_t s = (cudaStream_t)stream;
+    if ((rc = sign_all(p, s, p->d_sigs))) return rc;
+    return vote_and_report(p, s, report, h_outliers, outlier_cap, h_undecided, undecided_cap);
+}
+
+int scout_certify_host(scout_plan_t *p, const void *const *h_ptrs, scout_report_t *report,
+                       scout_outlier_t *h_outliers, uint64_t outlier_cap, uint64_t *h_undecided,
+                       uint64_t undecided_cap) {
+    if (!p || !h_ptrs || !report) return SCOUT_ERR_INVALID;
+    if ((outlier_cap && !h_outliers) || (undecided_cap && !h_undecided)) return SCOUT_ERR_INVALID;
+    const uint64_t n = (uint64_t)p->R * p->T;
+    for (uint64_t i = 0; i < n; ++i)
+        if (!h_ptrs[i]) return SCOUT_ERR_INVALID;
+    int rc = ensure_certify_buffers(p, outlier_cap, undecided_cap);
+    if (rc) return rc;
+    const uint64_t packed = p->tensor_poff[p->T];
+    if (!p->s_copy) {
+        SCOUT_CUDA(cudaStreamCreateWithFlags(&p->s_copy, cudaStreamNonBlocking));
+        SCOUT_CUDA(cudaStreamCreateWithFlags(&p->s_comp, cudaStreamNonBlocking));
+        for (int i = 0; i < 2; ++i) {
+            SCOUT_CUDA(cudaEventCreateWithFlags(&p->ev_copied[i], cudaEventDisableTiming));
+            SCOUT_CUDA(cudaEventCreateWithFlags(&p->ev_done[i], cudaEventDisableTiming));
+        }
+        p->stage_bytes = std::min<uint64_t>(packed, 256ull << 20);
+        p->stage_bytes = std::max<uint64_t>(p->stage_bytes, (uint64_t)p->tile_bytes + 256);
+        for (int i = 0; i < 2; ++i) SCOUT_CUDA(cudaMalloc(&p->d_stage[i], p->stage_bytes));
+    }
+    const uint64_t NT = p->tiles.size();
+    uint64_t slice = 0;
+    for (uint32_t r = 0; r < p->R; ++r) {
+        uint64_t t0 = 0;
+        while (t0 < NT) {
+            // largest run of tiles whose packed extent fits the staging buffer
+            const uint64_t a = p->tiles[t0].poff;
+            uint64_t t1 = t0;
+            while (t1 < NT && p->tiles[t1].poff + p->tiles[t1].nbytes - a <= p->stage_bytes) ++t1;
+            const uint64_t b = p->tiles[t1 - 1].poff + p->tiles[t1 - 1].nbytes;
+            const int buf = (int)(slice & 1);
+            if (slice >= 2) SCOUT_CUDA(cudaStreamWaitEvent(p->s_copy, p->ev_done[buf], 0));
+            for (uint32_t t = p->tiles[t0].tensor; t <= p->tiles[t1 - 1].tensor; ++t) {
+                const uint64_t lo = std::max<uint64_t>(a, p->tensor_poff[t]);
+                const uint64_t hi = std::min<uint64_t>(b, p->tensor_poff[t] + p->tensors[t].nbytes);
+                if (hi <= lo) continue;
+                const uint8_t *src = (const uint8_t *)h_ptrs[(uint64_t)r * p->T + t] + (lo - p->tensor_poff[t]);
+                SCOUT_CUDA(cudaMemcpyAsync(p->d_stage[buf] + (lo - a), src, hi - lo,
+                                           cudaMemcpyHostToDevice, p->s_copy));
+            }
+            SCOUT_CUDA(cudaEventRecord(p->ev_copied[buf], p->s_copy));
+            SCOUT_CUDA(cudaStreamWaitEvent(p->s_comp, p->ev_copied[buf], 0));
+            SignLaunch l;
+            l.tiles = p->d_tiles;
+            l.tile_begin = t0;
+            l.n_tiles = t1 - t0;
+            l.tiles_per_replica = NT;
+            l.replica_begin = r;
+            l.n_replicas = 1;
+            l.ptrs = nullptr;
+            l.T = p->T;
+            l.stage = p->d_stage[buf];
+            l.slice_begin = a;
+            l.recs = p->d_recs;
+            l.variant = p->variant;
+            l.grid = p->grid;
+            if ((rc = launch_sign_tiles(l, p->s_comp))) return rc;
+            SCOUT_CUDA(cudaEventRecord(p->ev_done[buf], p->s_comp));
+            t0 = t1;
+            ++slice;
+        }
+    }
+    rc = launch_finalize(p->d_chunks, p->chunks.size(), p->R, p->d_recs, NT, p->tile_bytes / ROW_BYTES,
+                         p->d_sigs, p->s_comp);
+    if (rc) return rc;
+    return vote_and_report(p, p->s_comp, report, h_outliers, outlier_cap, h_undecided, undecided_cap);
+}
+
+int scout_plan_results(const scout_plan_t *p, const scout_sig_t **d_sigs, const uint8_t **d_status,
+                       const uint64_t **d_bitmap) {
+    if (!p || !p->have_results) return SCOUT_ERR_INVALID;
+    if (d_sigs) *d_sigs = p->d_sigs;
+    if (d_status) *d_status = p->d_status;
+    if (d_bitmap) *d_bitmap = p->d_bitmap;
+    return SCOUT_OK;
+}
+
+int scout_plan_replica_bad_counts(const scout_plan_t *p, uint64_t *h_counts) {
+    if (!p || !h_counts || !p->have_results) return SCOUT_ERR_INVALID;
+    for (uint32_t r = 0; r < p->R; ++r) h_counts[r] = p->h_out->replica_bad[r];
+    return SCOUT_OK;
+}
+
+int scout_rollup_tensors(const scout_plan_t *p, const scout_sig_t *d_sigs, uint64_t *d_tensor_sigs,
+                         void *stream) {
+    if (!p || !d_sigs || !d_tensor_sigs) return SCOUT_ERR_INVALID;
+    return launch_rollup_tensors(p->d_chunks, p->d_tensor_chunk0, p->T, p->R, d_sigs, d_tensor_sigs,
+                                 (cudaStream_t)stream);
+}
+
+uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims) {
+    uint64_t a = mix64(SEED_SHAPE ^ (uint64_t)ndim);
+    for (uint32_t i = 0; i < ndim; ++i) a = mix64(a ^ dims[i]);
+    return a;
+}
+
+int scout_plan_set(scout_plan_t *p, const char *key, int64_t value) {
+    if (!p || !key) return SCOUT_ERR_INVALID;
+    if (!std::strcmp(key, "tile_bytes")) {
+        if (value < 2048 || value > 65536 || (value & (value - 1))) return SCOUT_ERR_INVALID;
+        if ((uint32_t)value == p->tile_bytes) return SCOUT_OK;
+        p->tile_bytes = (uint32_t)value;
+        try {
+            build_tiles(p);
+        } catch (const std::bad_alloc &) {
+            return SCOUT_ERR_NOMEM;
+        }
+        if (p->d_stage[0]) {  // staging was sized for the old tiles
+            for (int i = 0; i < 2; ++i) { cudaFree(p->d_stage[i]); p->d_stage[i] = nullptr; }
+            cudaStreamDestroy(p->s_copy);
+            cudaStreamDestroy(p->s_comp);
+            p->s_copy = p->s_comp = nullptr;
+            for (int i = 0; i < 2; ++i) {
+                cudaEventDestroy(p->ev_copied[i]);
+                cudaEventDestroy(p->ev_done[i]);
+                p->ev_copied[i] = p->ev_done[i] = nullptr;
+            }
+        }
+        return upload_tables(p);
+    }
+    if (!std::strcmp(key, "variant")) {
+        if (value < 0 || value > 1) return SCOUT_ERR_INVALID;
+        p->variant = (int)value;
+        return sign_grid_size(p->variant, p->device, &p->grid);
+    }
+    if (!std::strcmp(key, "grid")) {
+        if (value < 1 || value > 65535) return SCOUT_ERR_INVALID;
+        p->grid = (int)value;
+        return SCOUT_OK;
+    }
+    return SCOUT_ERR_INVALID;
+}
+
+int scout_plan_get(const scout_plan_t *p, const char *key, int64_t *value) {
+    if (!p || !key || !value) return SCOUT_ERR_INVALID;
+    if (!std::strcmp(key, "tile_bytes")) *value = p->tile_bytes;
+    else if (!std::strcmp(key, "variant")) *value = p->variant;
+    else if (!std::strcmp(key, "grid")) *value = p->grid;
+    else if (!std::strcmp(key, "n_tiles")) *value = (int64_t)p->tiles.size();
+    else if (!std::strcmp(key, "scratch_bytes")) *value = (int64_t)(p->tiles.size() * p->R * sizeof(TileRec));
+    else return SCOUT_ERR_INVALID;
+    return SCOUT_OK;
+}
+
+const char *scout_strerror(int code) {
+    switch (code) {
+        case SCOUT_OK: return "ok";
+        case SCOUT_ERR_INVALID: return "invalid argument";
+        case SCOUT_ERR_ALIGN: return "tensor address not 16-byte aligned";
+        case SCOUT_ERR_UNSUPPORTED: return "unsupported (more than 64 replicas, or a table too large)";
+        case SCOUT_ERR_CUDA: return "CUDA runtime error";
+        case SCOUT_ERR_NOMEM: return "out of memory";
+        case SCOUT_ERR_TRUNCATED: return "result list truncated (counters hold the true totals)";
+        default: return "unknown error";
+    }
+}
+
+int scout_version(void) { return 100; }
+
+const char *scout_last_cuda_error(void) { return g_last_cuda_error.c_str(); }
+
+}  // extern "C"

@@ -1,0 +1,145 @@
+// Internal declarations of the sm_100a sign+vote library (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "scout.h"
+
+namespace scout {
+
+// ---- SF64 signature constants ----------------------------------------------
+// The evidence of Sec. 5.2 is "a deterministic, position-sensitive 64-bit hash
+// over dtype, shape and bytes"; the function itself is left open there.  This
+// library's function: rows of 128 little-endian 32-bit words, row sum
+// S_q = sum_s m_s * w[128 q + s], h <- h * P + S_q, then a metadata mix.
+//   P   = floor(2^64 / golden ratio), G32 = floor(2^32 / golden ratio),
+//   MIX_A / MIX_B = fractional bits of sqrt 2 (made odd) / sqrt 3,
+//   SEED_* = fractional bits of sqrt 5, 7, 11, 13.
+constexpr uint64_t HASH_P = 0x9E3779B97F4A7C15ull;
+constexpr uint32_t HASH_G32 = 0x9E3779B9u;
+constexpr uint64_t MIX_A = 0x6A09E667F3BCC909ull;
+constexpr uint64_t MIX_B = 0xBB67AE8584CAA73Bull;
+constexpr uint64_t SEED_CHUNK = 0x3C6EF372FE94F82Bull;
+constexpr uint64_t SEED_TENSOR = 0xA54FF53A5F1D36F1ull;
+constexpr uint64_t SEED_SHAPE = 0x510E527FADE682D1ull;
+constexpr uint64_t SEED_CERT = 0x9B05688C2B3E6C1Full;
+constexpr uint32_t ROW_BYTES = 512;  // 128 words: one 16-byte vector per lane of a warp
+
+__host__ __device__ inline uint64_t mix64(uint64_t z) {
+    z ^= z >> 32;
+    z *= MIX_A;
+    z ^= z >> 29;
+    z *= MIX_B;
+    z ^= z >> 32;
+    return z;
+}
+
+// P^e mod 2^64 by square and multiply.
+__host__ __device__ inline uint64_t pow_p(uint64_t e) {
+    uint64_t r = 1, b = HASH_P;
+    while (e) {
+        if (e & 1) r *= b;
+        b *= b;
+        e >>= 1;
+    }
+    return r;
+}
+
+__host__ __device__ inline uint64_t finalize_hash(uint64_t h_raw, uint64_t nbytes, uint64_t k,
+                                                  uint32_t dtype, uint64_t meta) {
+    uint64_t t = mix64(SEED_CHUNK ^ nbytes);
+    t = mix64(t ^ k);
+    t = mix64(t ^ (uint64_t)dtype);
+    t = mix64(t ^ meta);
+    return mix64(h_raw + t);
+}
+
+// ---- device tables -----------------------------------------------------------
+// One work item of the scan: a run of whole rows of one chunk.
+struct TileDesc {
+    uint64_t off;     // byte offset inside the tensor
+    uint64_t poff;    // byte offset inside the packed (staged) image of one replica
+    uint32_t tensor;  // tensor index
+    uint32_t nbytes;  // bytes in this tile (<= tile_bytes; only a chunk's last tile is short)
+    uint32_t chunk;   // global chunk id
+    uint32_t dtype;   // SCOUT_DT_*
+};
+static_assert(sizeof(TileDesc) == 32, "TileDesc layout");
+
+struct ChunkDesc {
+    uint64_t nbytes;
+    uint64_t k;        // index of the chunk inside its tensor
+    uint64_t meta;     // caller's shape tag
+    uint64_t tile0;    // first tile of the chunk
+    uint32_t ntiles;
+    uint32_t dtype;
+    uint32_t tensor;
+    uint32_t pad;
+    uint64_t byte_offset;
+};
+static_assert(sizeof(ChunkDesc) == 56, "ChunkDesc layout");
+
+// Partial evidence of one (replica, tile).
+struct TileRec {
+    uint64_t h;       // sum over the tile's rows of P^(rows after it in the tile) * S_q
+    double sum, sumsq;
+    uint32_t nan_count, inf_count;
+};
+static_assert(sizeof(TileRec) == 32, "TileRec layout");
+
+// Results of the roll-up kernels, copied to the host by scout_certify.
+struct CertifyOut {
+    uint64_t counts[6];
+    uint64_t union_bitmap;
+    uint64_t certificate;
+    uint64_t replica_bad[64];
+};
+
+// ---- error plumbing ------------------------------------------------------------
+void set_cuda_error(cudaError_t e, const char *what);
+#define SCOUT_CUDA(call)                                  \
+    do {                                                  \
+        cudaError_t e__ = (call);                         \
+        if (e__ != cudaSuccess) {                         \
+            ::scout::set_cuda_error(e__, #call);          \
+            return SCOUT_ERR_CUDA;                        \
+        }                                                 \
+    } while (0)
+
+// ---- kernel launchers (defined in the .cu files) ------------------------------
+struct SignLaunch {
+    const TileDesc *tiles;        // device
+    uint64_t tile_begin;          // first tile of this launch
+    uint64_t n_tiles;             // tiles per replica in this launch
+    uint64_t tiles_per_replica;   // stride of the record array
+    uint32_t replica_begin;       // first replica of this launch
+    uint32_t n_replicas;          // replicas in this launch
+    const uint8_t *const *ptrs;   // device table [R][T], or nullptr in staged mode
+    uint64_t T;
+    const uint8_t *stage;         // staged mode: device image of packed bytes [slice_begin, ...)
+    uint64_t slice_begin;         // packed offset held at stage[0]
+    TileRec *recs;                // device [R][tiles_per_replica]
+    int variant;
+    int grid;                     // CTAs to launch
+};
+int launch_sign_tiles(const SignLaunch &a, cudaStream_t stream);
+int sign_grid_size(int variant, int device, int *grid);
+
+int launch_finalize(const ChunkDesc *chunks, uint64_t C, uint32_t R, const TileRec *recs,
+                    uint64_t tiles_per_replica, uint32_t tile_rows, scout_sig_t *d_sigs,
+                    cudaStream_t stream);
+
+int launch_vote(uint32_t R, uint64_t C, const scout_sig_t *d_sigs, uint8_t *d_status,
+                uint64_t *d_bitmap, scout_outlier_t *d_outliers, uint64_t outlier_cap,
+                uint64_t *d_undecided, uint64_t undecided_cap, uint64_t *d_counts,
+                uint64_t *d_majority, CertifyOut *d_out, cudaStream_t stream);
+int launch_certificate(uint64_t C, const uint64_t *d_majority, CertifyOut *d_out,
+                       cudaStream_t stream);
+int launch_rollup_tensors(const ChunkDesc *chunks, const uint64_t *tensor_chunk0, uint64_t T,
+                          uint32_t R, const scout_sig_t *d_sigs, uint64_t *d_tensor_sigs,
+                          cudaStream_t stream);
+
+}  // namespace scout

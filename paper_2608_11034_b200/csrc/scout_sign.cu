@@ -1,0 +1,402 @@
+// Comparable evidence (Sec. 5.2): the bulk fold of replica bytes into per-tile
+// partial records, and their finalisation into one record per (chunk, replica).
+//
+// Layout of the scan.  A row is 128 little-endian 32-bit words = 512 bytes =
+// one 16-byte vector per lane of a warp.  Lane l always holds words 4l..4l+3 of
+// a row, so its four slot multipliers m_{4l..4l+3} are loop constants, and the
+// row recurrence h <- h*P + S_q distributes over lanes: every lane runs its own
+// recurrence on its share of S_q and the shares are added once per tile
+// (integer addition mod 2^64 is order-free).  The fp64 sums use a fixed
+// lane -> element mapping and a fixed butterfly, so results are bitwise
+// reproducible.
+//
+// Non-finite values.  The hot loop does not classify elements.  Every finite
+// fp32/bf16/fp16 square is below 2^256 and every non-finite element pushes the
+// naive sum of squares to at least 2^256 (or NaN), so "!(sumsq < 2^256)" is a
+// necessary condition for a non-finite element in the tile.  A tile that trips
+// it is scanned again (it is still in L2) by a loop that classifies every
+// element, counts NaN/Inf and sums the finite ones only.
+#include <cuda_fp16.h>
+
+#include "scout_internal.h"
+
+namespace scout {
+namespace {
+
+constexpr int SIGN_THREADS = 256;
+constexpr int UNROLL = 4;
+
+struct Acc {
+    double s0, s1, q0, q1;
+};
+
+__device__ __forceinline__ uint4 ld_stream16(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// 16 bytes at tile[byte_off..], bytes at or past nbytes read as zero.  Only
+// the last row of a chunk can be ragged, so the byte loop is off the hot path.
+__device__ __noinline__ uint4 ld_masked16(const uint8_t *tile, uint32_t byte_off, uint32_t nbytes) {
+    uint32_t w[4] = {0u, 0u, 0u, 0u};
+    if (byte_off + 16u <= nbytes) {
+        uint4 v = ld_stream16(tile + byte_off);
+        return v;
+    }
+    if (byte_off < nbytes) {
+        uint32_t n = nbytes - byte_off;
+        for (uint32_t i = 0; i < n; ++i) w[i >> 2] |= (uint32_t)tile[byte_off + i] << (8u * (i & 3u));
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+__device__ __forceinline__ void acc2(Acc &a, double x0, double x1) {
+    a.s0 += x0;
+    a.q0 = fma(x0, x0, a.q0);
+    a.s1 += x1;
+    a.q1 = fma(x1, x1, a.q1);
+}
+
+// ---- per-dtype element paths: fast (no classification) -----------------------
+template <int DT>
+__device__ __forceinline__ void stats_fast(const uint4 &v, Acc &a) {
+    if constexpr (DT == SCOUT_DT_F32) {
+        acc2(a, (double)__uint_as_float(v.x), (double)__uint_as_float(v.y));
+        acc2(a, (double)__uint_as_float(v.z), (double)__uint_as_float(v.w));
+    } else if constexpr (DT == SCOUT_DT_BF16) {
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            acc2(a, (double)__uint_as_float(w[i] << 16), (double)__uint_as_float(w[i] & 0xFFFF0000u));
+    } else if constexpr (DT == SCOUT_DT_F16) {
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
+            acc2(a, (double)f.x, (double)f.y);
+        }
+    } else if constexpr (DT == SCOUT_DT_F64) {
+        acc2(a, __hiloint2double((int)v.y, (int)v.x), __hiloint2double((int)v.w, (int)v.z));
+    } else if constexpr (DT == SCOUT_DT_I64) {
+        acc2(a, (double)(long long)(((uint64_t)v.y << 32) | v.x),
+             (double)(long long)(((uint64_t)v.w << 32) | v.z));
+    } else if constexpr (DT == SCOUT_DT_I32) {
+        acc2(a, (double)(int)v.x, (double)(int)v.y);
+        acc2(a, (double)(int)v.z, (double)(int)v.w);
+    }
+}
+
+template <int DT>
+__device__ __forceinline__ bool may_hold_nonfinite(const Acc &a) {
+    if constexpr (DT == SCOUT_DT_F32 || DT == SCOUT_DT_BF16 || DT == SCOUT_DT_F16) {
+        return !(a.q0 + a.q1 < 1.157920892373162e77);  // 2^256
+    } else if constexpr (DT == SCOUT_DT_F64) {
+        return !(a.q0 + a.q1 < __longlong_as_double(0x7FF0000000000000ll));
+    } else {
+        return false;
+    }
+}
+
+// ---- per-dtype element paths: classifying (slow) ------------------------------
+struct SlowAcc {
+    double s, q;
+    uint32_t nan_count, inf_count;
+};
+
+__device__ __forceinline__ void slow_add(SlowAcc &a, double x, bool nonfinite, bool is_nan) {
+    if (nonfinite) {
+        if (is_nan) ++a.nan_count; else ++a.inf_count;
+    } else {
+        a.s += x;
+        a.q = fma(x, x, a.q);
+    }
+}
+
+template <int DT>
+__device__ __forceinline__ void stats_slow(const uint4 &v, SlowAcc &a) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    if constexpr (DT == SCOUT_DT_F32) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            slow_add(a, (double)__uint_as_float(w[i]), (w[i] & 0x7F800000u) == 0x7F800000u,
+                     (w[i] & 0x007FFFFFu) != 0u);
+    } else if constexpr (DT == SCOUT_DT_BF16) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint32_t lo = w[i] << 16, hi = w[i] & 0xFFFF0000u;
+            slow_add(a, (double)__uint_as_float(lo), (lo & 0x7F800000u) == 0x7F800000u, (lo & 0x007F0000u) != 0u);
+            slow_add(a, (double)__uint_as_float(hi), (hi & 0x7F800000u) == 0x7F800000u, (hi & 0x007F0000u) != 0u);
+        }
+    } else if constexpr (DT == SCOUT_DT_F16) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
+            uint32_t lo = w[i] & 0xFFFFu, hi = w[i] >> 16;
+            slow_add(a, (double)f.x, (lo & 0x7C00u) == 0x7C00u, (lo & 0x03FFu) != 0u);
+            slow_add(a, (double)f.y, (hi & 0x7C00u) == 0x7C00u, (hi & 0x03FFu) != 0u);
+        }
+    } else if constexpr (DT == SCOUT_DT_F64) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            uint32_t lo = w[2 * i], hi = w[2 * i + 1];
+            slow_add(a, __hiloint2double((int)hi, (int)lo), (hi & 0x7FF00000u) == 0x7FF00000u,
+                     ((hi & 0x000FFFFFu) | lo) != 0u);
+        }
+    }
+}
+
+template <int DT>
+__device__ __noinline__ void rescan_classifying(const uint8_t *tile, uint32_t nbytes, uint32_t lane,
+                                                double &sum, double &sumsq, uint32_t &nan_count,
+                                                uint32_t &inf_count) {
+    SlowAcc a = {0.0, 0.0, 0u, 0u};
+    const uint32_t rows = (nbytes + ROW_BYTES - 1) / ROW_BYTES;
+    for (uint32_t row = 0; row < rows; ++row) {
+        uint4 v = ld_masked16(tile, row * ROW_BYTES + 16u * lane, nbytes);
+        stats_slow<DT>(v, a);
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        a.s += __shfl_xor_sync(0xFFFFFFFFu, a.s, d);
+        a.q += __shfl_xor_sync(0xFFFFFFFFu, a.q, d);
+        a.nan_count += __shfl_xor_sync(0xFFFFFFFFu, a.nan_count, d);
+        a.inf_count += __shfl_xor_sync(0xFFFFFFFFu, a.inf_count, d);
+    }
+    sum = a.s;
+    sumsq = a.q;
+    nan_count = a.nan_count;
+    inf_count = a.inf_count;
+}
+
+__device__ __forceinline__ void fold_row(uint64_t &h, const uint4 &v, const uint32_t (&m)[4]) {
+    uint64_t s = (uint64_t)m[0] * v.x;
+    s += (uint64_t)m[1] * v.y;
+    s += (uint64_t)m[2] * v.z;
+    s += (uint64_t)m[3] * v.w;
+    h = h * HASH_P + s;
+}
+
+// One warp scans one tile with direct 16-byte loads.
+template <int DT>
+__device__ __forceinline__ void scan_tile(const uint8_t *tile, uint32_t nbytes, uint32_t lane,
+                                          TileRec &out) {
+    uint32_t m[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) m[j] = ((4u * lane + j + 1u) * HASH_G32) | 1u;
+
+    const uint32_t full = nbytes / ROW_BYTES;
+    const uint8_t *p = tile + 16u * lane;
+    uint64_t h = 0;
+    Acc a = {0.0, 0.0, 0.0, 0.0};
+    uint32_t row = 0;
+    for (; row + UNROLL <= full; row += UNROLL) {
+        uint4 v[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) v[u] = ld_stream16(p + (size_t)(row + u) * ROW_BYTES);
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            fold_row(h, v[u], m);
+            stats_fast<DT>(v[u], a);
+        }
+    }
+    for (; row < full; ++row) {
+        uint4 v = ld_stream16(p + (size_t)row * ROW_BYTES);
+        fold_row(h, v, m);
+        stats_fast<DT>(v, a);
+    }
+    if (nbytes % ROW_BYTES) {  // ragged last row of a chunk: missing words are zero
+        uint4 v = ld_masked16(tile, full * ROW_BYTES + 16u * lane, nbytes);
+        fold_row(h, v, m);
+        stats_fast<DT>(v, a);
+    }
+
+    double s = a.s0 + a.s1, q = a.q0 + a.q1;
+    const bool suspect = __any_sync(0xFFFFFFFFu, may_hold_nonfinite<DT>(a));
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        h += __shfl_xor_sync(0xFFFFFFFFu, h, d);
+        s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
+        q += __shfl_xor_sync(0xFFFFFFFFu, q, d);
+    }
+    uint32_t nan_count = 0, inf_count = 0;
+    if constexpr (DT == SCOUT_DT_F32 || DT == SCOUT_DT_BF16 || DT == SCOUT_DT_F16 ||
+                  DT == SCOUT_DT_F64) {
+        if (suspect) rescan_classifying<DT>(tile, nbytes, lane, s, q, nan_count, inf_count);
+    }
+    out.h = h;
+    out.sum = s;
+    out.sumsq = q;
+    out.nan_count = nan_count;
+    out.inf_count = inf_count;
+}
+
+struct SignArgs {
+    const TileDesc *tiles;
+    uint64_t tile_begin, n_tiles, tiles_per_replica;
+    uint32_t replica_begin, n_replicas;
+    const uint8_t *const *ptrs;
+    uint64_t T;
+    const uint8_t *stage;
+    uint64_t slice_begin;
+    TileRec *recs;
+};
+
+__device__ __forceinline__ void scan_dispatch(uint32_t dtype, const uint8_t *tile, uint32_t nbytes,
+                                              uint32_t lane, TileRec &rec) {
+    switch (dtype) {
+        case SCOUT_DT_F32:  scan_tile<SCOUT_DT_F32>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_BF16: scan_tile<SCOUT_DT_BF16>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_I64:  scan_tile<SCOUT_DT_I64>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_F16:  scan_tile<SCOUT_DT_F16>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_F64:  scan_tile<SCOUT_DT_F64>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_I32:  scan_tile<SCOUT_DT_I32>(tile, nbytes, lane, rec); break;
+        default:            scan_tile<SCOUT_DT_U8>(tile, nbytes, lane, rec); break;
+    }
+}
+
+// Persistent grid; every warp takes whole tiles, replica-major, round-robin.
+__global__ void __launch_bounds__(SIGN_THREADS) sign_tiles_direct(const SignArgs a) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint64_t warp = (uint64_t)blockIdx.x * (SIGN_THREADS / 32) + (threadIdx.x >> 5);
+    const uint64_t n_warps = (uint64_t)gridDim.x * (SIGN_THREADS / 32);
+    const uint64_t n_items = a.n_tiles * a.n_replicas;
+    for (uint64_t item = warp; item < n_items; item += n_warps) {
+        const uint32_t rr = (uint32_t)(item / a.n_tiles);
+        const uint64_t t = a.tile_begin + (item - (uint64_t)rr * a.n_tiles);
+        const uint32_t r = a.replica_begin + rr;
+        const TileDesc td = a.tiles[t];
+        const uint8_t *tile = a.ptrs ? a.ptrs[(uint64_t)r * a.T + td.tensor] + td.off
+                                     : a.stage + (td.poff - a.slice_begin);
+        TileRec rec;
+        scan_dispatch(td.dtype, tile, td.nbytes, lane, rec);
+        if (lane == 0) {
+            uint4 *dst = reinterpret_cast<uint4 *>(&a.recs[(uint64_t)r * a.tiles_per_replica + t]);
+            dst[0] = make_uint4((uint32_t)rec.h, (uint32_t)(rec.h >> 32),
+                                (uint32_t)__double2loint(rec.sum), (uint32_t)__double2hiint(rec.sum));
+            dst[1] = make_uint4((uint32_t)__double2loint(rec.sumsq), (uint32_t)__double2hiint(rec.sumsq),
+                                rec.nan_count, rec.inf_count);
+        }
+    }
+}
+
+// ---- finalise: tile partials -> one record per (chunk, replica) --------------
+// Segment combine: for a split after some rows, H_raw = H_raw(left) * P^(rows
+// right) + H_raw(right).  A lane walks tiles lane, lane+32, ... with the
+// multiplier P^(32 * tile_rows), then weights its value by the rows that follow
+// its last tile; the chunk's last tile (the only one that can be short) is added
+// with weight one; the lane values add up to H_raw.  The fp64 partials are added
+// per lane in ascending tile order and then through a fixed butterfly.
+constexpr int FIN_THREADS = 128;
+
+__global__ void __launch_bounds__(FIN_THREADS) finalize_chunks(const ChunkDesc *chunks, uint64_t C,
+                                                               uint32_t R, const TileRec *recs,
+                                                               uint64_t tiles_per_replica,
+                                                               uint32_t tile_rows, uint64_t p_stride,
+                                                               scout_sig_t *sigs) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint64_t warp = (uint64_t)blockIdx.x * (FIN_THREADS / 32) + (threadIdx.x >> 5);
+    const uint64_t n_warps = (uint64_t)gridDim.x * (FIN_THREADS / 32);
+    for (uint64_t item = warp; item < C * R; item += n_warps) {
+        const uint64_t c = item / R;
+        const uint32_t r = (uint32_t)(item - c * R);
+        const ChunkDesc cd = chunks[c];
+        const TileRec *tr = recs + (uint64_t)r * tiles_per_replica + cd.tile0;
+        const uint32_t nt = cd.ntiles;
+        const uint64_t rows_total = (cd.nbytes + ROW_BYTES - 1) / ROW_BYTES;
+        const uint64_t rows_last = rows_total - (uint64_t)(nt - 1) * tile_rows;
+
+        uint64_t h = 0;
+        double s = 0.0, q = 0.0;
+        uint32_t nan_count = 0, inf_count = 0, last_t = 0;
+        const uint32_t n_full = nt - 1;  // every tile but the chunk's last has tile_rows rows
+        for (uint32_t t = lane; t < n_full; t += 32) {
+            const TileRec x = tr[t];
+            h = h * p_stride + x.h;
+            s += x.sum;
+            q += x.sumsq;
+            nan_count += x.nan_count;
+            inf_count += x.inf_count;
+            last_t = t;
+        }
+        if (lane < n_full) h *= pow_p(rows_last + (uint64_t)tile_rows * (n_full - 1 - last_t));
+        if (lane == (n_full & 31u)) {  // the last (possibly short) tile: nothing follows it
+            const TileRec x = tr[n_full];
+            h += x.h;
+            s += x.sum;
+            q += x.sumsq;
+            nan_count += x.nan_count;
+            inf_count += x.inf_count;
+        }
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) {
+            h += __shfl_xor_sync(0xFFFFFFFFu, h, d);
+            s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
+            q += __shfl_xor_sync(0xFFFFFFFFu, q, d);
+            nan_count += __shfl_xor_sync(0xFFFFFFFFu, nan_count, d);
+            inf_count += __shfl_xor_sync(0xFFFFFFFFu, inf_count, d);
+        }
+        if (lane == 0) {
+            scout_sig_t o;
+            o.hash = finalize_hash(h, cd.nbytes, cd.k, cd.dtype, cd.meta);
+            o.nan_count = nan_count;
+            o.inf_count = inf_count;
+            o.sum = s;
+            o.sumsq = q;
+            sigs[c * R + r] = o;
+        }
+    }
+}
+
+}  // namespace
+
+int sign_grid_size(int variant, int device, int *grid) {
+    int sms = 0, per_sm = 0;
+    SCOUT_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+    (void)variant;
+    SCOUT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sign_tiles_direct, SIGN_THREADS, 0));
+    if (per_sm < 1) per_sm = 1;
+    *grid = sms * per_sm;
+    return SCOUT_OK;
+}
+
+int launch_sign_tiles(const SignLaunch &l, cudaStream_t stream) {
+    if (l.n_tiles == 0 || l.n_replicas == 0) return SCOUT_OK;
+    SignArgs a;
+    a.tiles = l.tiles;
+    a.tile_begin = l.tile_begin;
+    a.n_tiles = l.n_tiles;
+    a.tiles_per_replica = l.tiles_per_replica;
+    a.replica_begin = l.replica_begin;
+    a.n_replicas = l.n_replicas;
+    a.ptrs = l.ptrs;
+    a.T = l.T;
+    a.stage = l.stage;
+    a.slice_begin = l.slice_begin;
+    a.recs = l.recs;
+    const uint64_t items = l.n_tiles * l.n_replicas;
+    const uint64_t want = (items + SIGN_THREADS / 32 - 1) / (SIGN_THREADS / 32);
+    int grid = l.grid;
+    if ((uint64_t)grid > want) grid = (int)want;
+    sign_tiles_direct<<<grid, SIGN_THREADS, 0, stream>>>(a);
+    SCOUT_CUDA(cudaGetLastError());
+    return SCOUT_OK;
+}
+
+int launch_finalize(const ChunkDesc *chunks, uint64_t C, uint32_t R, const TileRec *recs,
+                    uint64_t tiles_per_replica, uint32_t tile_rows, scout_sig_t *d_sigs,
+                    cudaStream_t stream) {
+    if (C == 0) return SCOUT_OK;
+    const uint64_t items = C * R;
+    uint64_t blocks = (items + FIN_THREADS / 32 - 1) / (FIN_THREADS / 32);
+    if (blocks > 148ull * 16) blocks = 148ull * 16;
+    finalize_chunks<<<(int)blocks, FIN_THREADS, 0, stream>>>(chunks, C, R, recs, tiles_per_replica,
+                                                            tile_rows, pow_p(32ull * tile_rows),
+                                                            d_sigs);
+    SCOUT_CUDA(cudaGetLastError());
+    return SCOUT_OK;
+}
+
+}  // namespace scout

@@ -1,0 +1,188 @@
+// Exact consensus (Sec. 5.3; Algorithm 1, Exact branch) over the gathered
+// evidence of every chunk, the compaction of disagreements into lists, and the
+// roll-ups built on top of it.
+#include "scout_internal.h"
+
+namespace scout {
+namespace {
+
+constexpr int VOTE_THREADS = 256;
+
+// One warp per chunk.  Lane j holds e_j and e_{j+32}.  cnt_j = #{i : e_i = e_j};
+// c* = max cnt.  2 c* <= R: Inconclusive, bitmap 0.  Otherwise e* is the unique
+// value with count c*, bit j = 1{e_j != e*}.  Outlier pairs and undecided chunk
+// ids are appended with one atomic per warp.
+__global__ void __launch_bounds__(VOTE_THREADS) vote_chunks(
+    uint32_t R, uint64_t C, const scout_sig_t *__restrict__ sigs, uint8_t *status_out,
+    uint64_t *bitmap_out, scout_outlier_t *outliers, uint64_t outlier_cap, uint64_t *undecided,
+    uint64_t undecided_cap, uint64_t *counts, uint64_t *majority_out, CertifyOut *cert) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint64_t warp = (uint64_t)blockIdx.x * (VOTE_THREADS / 32) + (threadIdx.x >> 5);
+    const uint64_t n_warps = (uint64_t)gridDim.x * (VOTE_THREADS / 32);
+    uint32_t n_agree = 0, n_attr = 0, n_inc = 0;  // per warp, identical in all lanes
+    uint64_t union_bits = 0;
+
+    for (uint64_t c = warp; c < C; c += n_warps) {
+        const scout_sig_t *e = sigs + c * R;
+        const bool have0 = lane < R, have1 = lane + 32u < R;
+        const uint64_t e0 = have0 ? e[lane].hash : 0ull;
+        const uint64_t e1 = have1 ? e[lane + 32u].hash : 0ull;
+        uint32_t cnt0 = 0, cnt1 = 0;
+        for (uint32_t i = 0; i < R; ++i) {
+            const uint64_t lo = __shfl_sync(0xFFFFFFFFu, e0, i & 31u);
+            const uint64_t hi = __shfl_sync(0xFFFFFFFFu, e1, i & 31u);
+            const uint64_t ei = i < 32u ? lo : hi;
+            cnt0 += (ei == e0);
+            cnt1 += (ei == e1);
+        }
+        if (!have0) cnt0 = 0;
+        if (!have1) cnt1 = 0;
+        const uint32_t mine = cnt0 > cnt1 ? cnt0 : cnt1;
+        const uint32_t best = __reduce_max_sync(0xFFFFFFFFu, mine);
+
+        uint64_t bitmap = 0, majority = 0;
+        uint32_t st;
+        if (2u * best <= R) {
+            st = SCOUT_INCONCLUSIVE;
+            ++n_inc;
+        } else {
+            // the lanes holding e* (count == best) agree on one value
+            const uint32_t holders = __ballot_sync(0xFFFFFFFFu, cnt0 == best);
+            const uint32_t holders_hi = __ballot_sync(0xFFFFFFFFu, cnt1 == best);
+            if (holders) majority = __shfl_sync(0xFFFFFFFFu, e0, __ffs(holders) - 1);
+            else         majority = __shfl_sync(0xFFFFFFFFu, e1, __ffs(holders_hi) - 1);
+            const uint32_t b0 = __ballot_sync(0xFFFFFFFFu, have0 && e0 != majority);
+            const uint32_t b1 = __ballot_sync(0xFFFFFFFFu, have1 && e1 != majority);
+            bitmap = ((uint64_t)b1 << 32) | b0;
+            st = bitmap ? SCOUT_ATTRIBUTED : SCOUT_AGREE;
+            if (bitmap) ++n_attr; else ++n_agree;
+            union_bits |= bitmap;
+        }
+        if (lane == 0) {
+            if (status_out) status_out[c] = (uint8_t)st;
+            if (bitmap_out) bitmap_out[c] = bitmap;
+            if (majority_out) majority_out[c] = majority;
+        }
+        if (bitmap) {  // warp-aggregated append of (chunk, replica) pairs
+            const uint32_t n = __popcll(bitmap);
+            unsigned long long base = 0;
+            if (lane == 0) base = atomicAdd((unsigned long long *)&counts[4], (unsigned long long)n);
+            base = __shfl_sync(0xFFFFFFFFu, base, 0);
+            const uint32_t b0 = (uint32_t)bitmap, b1 = (uint32_t)(bitmap >> 32);
+            const uint32_t below = (1u << lane) - 1u;
+            if ((b0 >> lane) & 1u) {
+                const uint64_t pos = base + __popc(b0 & below);
+                if (pos < outlier_cap) outliers[pos] = scout_outlier_t{c, lane, 0u};
+            }
+            if ((b1 >> lane) & 1u) {
+                const uint64_t pos = base + __popc(b0) + __popc(b1 & below);
+                if (pos < outlier_cap) outliers[pos] = scout_outlier_t{c, lane + 32u, 0u};
+            }
+            if (cert && lane == 0) {
+                uint64_t b = bitmap;
+                while (b) {
+                    const int j = __ffsll((long long)b) - 1;
+                    atomicAdd((unsigned long long *)&cert->replica_bad[j], 1ull);
+                    b &= b - 1;
+                }
+            }
+        }
+        if (st == SCOUT_INCONCLUSIVE && lane == 0) {
+            const unsigned long long pos = atomicAdd((unsigned long long *)&counts[5], 1ull);
+            if (pos < undecided_cap) undecided[pos] = c;
+        }
+    }
+
+    // block-level aggregation of the status counters: one atomic per counter per CTA
+    __shared__ uint32_t sh[3];
+    __shared__ unsigned long long sh_union;
+    if (threadIdx.x == 0) { sh[0] = sh[1] = sh[2] = 0u; sh_union = 0ull; }
+    __syncthreads();
+    if (lane == 0) {
+        if (n_agree) atomicAdd(&sh[0], n_agree);
+        if (n_attr) atomicAdd(&sh[1], n_attr);
+        if (n_inc) atomicAdd(&sh[2], n_inc);
+        if (union_bits) atomicOr(&sh_union, (unsigned long long)union_bits);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (sh[0]) atomicAdd((unsigned long long *)&counts[1], (unsigned long long)sh[0]);
+        if (sh[1]) atomicAdd((unsigned long long *)&counts[2], (unsigned long long)sh[1]);
+        if (sh[2]) atomicAdd((unsigned long long *)&counts[3], (unsigned long long)sh[2]);
+        if (cert && sh_union) atomicOr((unsigned long long *)&cert->union_bitmap, sh_union);
+        if (blockIdx.x == 0) counts[0] = C;
+    }
+}
+
+// Certificate: a <- mix64(seed ^ C); a <- mix64(a ^ majority_c) for every chunk
+// in order.  The chain is sequential by construction; one warp streams the
+// hashes in coalesced groups of 32 and lane 0 runs the chain.
+__global__ void certificate_chain(uint64_t C, const uint64_t *__restrict__ majority, CertifyOut *out) {
+    const uint32_t lane = threadIdx.x;
+    uint64_t a = mix64(SEED_CERT ^ C);
+    uint64_t next = lane < C ? majority[lane] : 0ull;
+    for (uint64_t base = 0; base < C; base += 32) {
+        const uint64_t cur = next;
+        const uint64_t nb = base + 32 + lane;
+        next = nb < C ? majority[nb] : 0ull;
+        const uint32_t n = (uint32_t)((C - base) < 32 ? (C - base) : 32);
+        for (uint32_t i = 0; i < n; ++i) {
+            const uint64_t hsh = __shfl_sync(0xFFFFFFFFu, cur, i);
+            a = mix64(a ^ hsh);
+        }
+    }
+    if (lane == 0) {
+        out->certificate = out->counts[3] ? 0ull : a;
+    }
+}
+
+// Tensor-level signature (the granularity of Sec. 5.2): chunk hashes of one
+// (tensor, replica) folded in order.  One thread per (tensor, replica).
+__global__ void rollup_tensors(const uint64_t *__restrict__ tensor_chunk0, uint64_t T, uint32_t R,
+                               const scout_sig_t *__restrict__ sigs, uint64_t *out) {
+    const uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= T * R) return;
+    const uint64_t t = i / R;
+    const uint32_t r = (uint32_t)(i - t * R);
+    const uint64_t c0 = tensor_chunk0[t], c1 = tensor_chunk0[t + 1];
+    uint64_t a = mix64(SEED_TENSOR ^ (c1 - c0));
+    for (uint64_t c = c0; c < c1; ++c) a = mix64(a ^ sigs[c * R + r].hash);
+    out[i] = a;
+}
+
+}  // namespace
+
+int launch_vote(uint32_t R, uint64_t C, const scout_sig_t *d_sigs, uint8_t *d_status,
+                uint64_t *d_bitmap, scout_outlier_t *d_outliers, uint64_t outlier_cap,
+                uint64_t *d_undecided, uint64_t undecided_cap, uint64_t *d_counts,
+                uint64_t *d_majority, CertifyOut *d_out, cudaStream_t stream) {
+    if (d_out) SCOUT_CUDA(cudaMemsetAsync(d_out, 0, sizeof(CertifyOut), stream));
+    if ((void *)d_counts != (void *)d_out)
+        SCOUT_CUDA(cudaMemsetAsync(d_counts, 0, 6 * sizeof(uint64_t), stream));
+    uint64_t blocks = (C + VOTE_THREADS / 32 - 1) / (VOTE_THREADS / 32);
+    if (blocks > 148ull * 8) blocks = 148ull * 8;
+    if (blocks == 0) blocks = 1;
+    vote_chunks<<<(int)blocks, VOTE_THREADS, 0, stream>>>(R, C, d_sigs, d_status, d_bitmap, d_outliers,
+                                                         outlier_cap, d_undecided, undecided_cap,
+                                                         d_counts, d_majority, d_out);
+    SCOUT_CUDA(cudaGetLastError());
+    return SCOUT_OK;
+}
+
+int launch_certificate(uint64_t C, const uint64_t *d_majority, CertifyOut *d_out, cudaStream_t stream) {
+    certificate_chain<<<1, 32, 0, stream>>>(C, d_majority, d_out);
+    SCOUT_CUDA(cudaGetLastError());
+    return SCOUT_OK;
+}
+
+int launch_rollup_tensors(const ChunkDesc *, const uint64_t *tensor_chunk0, uint64_t T, uint32_t R,
+                          const scout_sig_t *d_sigs, uint64_t *d_tensor_sigs, cudaStream_t stream) {
+    const uint64_t n = T * R;
+    if (n == 0) return SCOUT_OK;
+    rollup_tensors<<<(unsigned)((n + 127) / 128), 128, 0, stream>>>(tensor_chunk0, T, R, d_sigs,
+                                                                   d_tensor_sigs);
+    SCOUT_CUDA(cudaGetLastError());
+    return SCOUT_OK;
+}
+
+}  // namespace scout

@@ -38,7 +38,7 @@ class TensorSpec:
     name: str
     shape: Tuple[int, ...]
     dtype: str                  # key of DTYPE_BYTES
-    dist: str                   # "normal" | "absnormal" | "randint40" | "bytes"
+    dist: str                   # "normal" | "absnormal" | "randint40" | "randfull" | "bytes"
     std: float = 1.0
 
     @property
@@ -207,6 +207,8 @@ def _fill(view: torch.Tensor, spec: TensorSpec, gen: torch.Generator) -> None:
         view.abs_()
     elif spec.dist == "randint40":
         view.random_(0, 1 << 40, generator=gen)
+    elif spec.dist == "randfull":
+        view.random_(generator=gen)
     elif spec.dist == "bytes":
         view.random_(0, 256, generator=gen)
     else:

@@ -57,3 +57,59 @@ def expected_from_patches(w, chunks):
             undecided.append(c)
         outliers += [(c, r) for r in range(w.R) if (B >> r) & 1]
     return sorted(outliers), undecided
+
+
+# ---- CUDA path plumbing (imported lazily so CPU-only runs never load it) -----
+
+def gpu_plan(w, chunk_bytes=None, tags=None, tile_bytes=None):
+    from paper_2608_11034_b200 import binding
+    tags = shape_tags(w) if tags is None else tags
+    plan = binding.Plan(w.R, binding.make_tensor_table(w.specs, tags),
+                        w.chunk_bytes if chunk_bytes is None else chunk_bytes)
+    if tile_bytes is not None:
+        binding.scout_plan_set(plan.handle, "tile_bytes", tile_bytes)
+    return plan
+
+
+def gpu_sign_vote(w, views, chunk_bytes=None, tags=None, tile_bytes=None, caps=(4096, 4096)):
+    """-> fetch() dict of the CUDA path over device-resident views[r][t]."""
+    plan = gpu_plan(w, chunk_bytes, tags, tile_bytes)
+    plan.bind(views)
+    plan.sign_and_vote(*caps)
+    out = plan.fetch()
+    plan.close()
+    return out
+
+
+def chunk_abs_sums(w, views, chunks):
+    """sum |x| over the finite elements of every (chunk, replica): the scale of
+    the tolerance on the sums."""
+    out = np.zeros((len(chunks), w.R))
+    for r in range(w.R):
+        host = [inputs.to_numpy_bytes(v) for v in views[r]]
+        for c, ch in enumerate(chunks):
+            dt = w.specs[int(ch["tensor"])].dtype
+            if dt == "u8":
+                continue
+            b = host[int(ch["tensor"])][int(ch["byte_offset"]):int(ch["byte_offset"] + ch["nbytes"])]
+            x = np.abs(defn.values_f64(b.tobytes(), dt))
+            out[c, r] = x[np.isfinite(x)].sum()
+    return out
+
+
+REL_TOL = 1e-12
+
+
+def assert_sigs_match(gpu_sigs, orc_sigs, abs_sums):
+    """Bit-exact hashes and counts; sums within 1e-12 of the un-cancelled scale
+    (|d sum| <= 1e-12 * sum|x|, |d sumsq| <= 1e-12 * sumsq)."""
+    assert gpu_sigs.shape == orc_sigs.shape
+    assert (gpu_sigs["hash"] == orc_sigs["hash"]).all()
+    assert (gpu_sigs["nan_count"] == orc_sigs["nan_count"]).all()
+    assert (gpu_sigs["inf_count"] == orc_sigs["inf_count"]).all()
+    for name, scale in (("sum", abs_sums), ("sumsq", np.abs(orc_sigs["sumsq"]))):
+        g, o = gpu_sigs[name], orc_sigs[name]
+        both_inf = np.isinf(g) & np.isinf(o) & (np.sign(g) == np.sign(o))
+        err = np.where(both_inf, 0.0, np.abs(g - o))
+        assert np.isfinite(err).all(), name
+        assert (err <= REL_TOL * scale).all(), (name, float(err.max()))
