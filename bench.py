@@ -1,0 +1,428 @@
+#!/usr/bin/env python
+"""Throughput of the sign+vote hot path on seeded synthetic replica sets.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl reference]
+
+One step = one pass of the whole hot path over one replica set: chunk
+signatures for every replica, strict-majority vote, compaction and (config 4)
+the certify roll-up.  The metric is GB/s of replica data scanned.  Prints ONE
+JSON line on rank 0.
+
+  value         inputs resident in HBM, CUDA-event time over exactly K steps
+  e2e           the same metric through scout_certify_host: replicas in pinned
+                HOST memory, host->device copies inside the timed region
+  roofline      the scan kernel alone (in-stream CUDA events inside the library)
+                against the measured HBM copy bandwidth
+  cpu_baseline  the CPU oracle, as it stands, on a bounded sample of the workload
+
+With N > 1 every rank scans its own replica set (no data-path collective):
+weak scaling, value = bytes of all ranks / max-over-ranks time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "replica GB/s scanned (sign+vote)"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes per algorithmic byte of the scan kernel, from the ncu capture
+# summarised in profiles/ (None until a capture exists)
+SCAN_TRAFFIC_RATIO = None
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=4, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--scale", type=float, default=1.0, help="shrink the workload (debugging only)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--variant", type=int, default=None)
+    ap.add_argument("--tile-bytes", type=int, default=None)
+    return ap.parse_args()
+
+
+# ------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.path = tempfile.mktemp(suffix=".csv")
+        self.proc = None
+        try:
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        try:
+            os.unlink(self.path)
+        except OSError:
+            pass
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "power_w_max": max(pw),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------ CPU oracle legs
+
+def oracle_sample(w, views, chunk_bytes, budget_bytes):
+    """Whole leading chunks of replica 0's tensors, up to budget_bytes, as host
+    arrays plus the matching tensor table (same dtype and shape tag, so the
+    records are those of the full workload's chunks)."""
+    from oracle import scout_oracle as orc
+    from paper_2608_11034_b200 import inputs
+    code = {"u8": 0, "f32": 1, "bf16": 2, "i64": 3, "f16": 4, "f64": 5, "i32": 6}
+    per_tensor = max(chunk_bytes, budget_bytes // len(w.specs) // chunk_bytes * chunk_bytes)
+    rows, arrays, picked, total = [], [], [], 0
+    for t, s in enumerate(w.specs):
+        if total >= budget_bytes:
+            break
+        n = min(s.nbytes, per_tensor)
+        if n < s.nbytes:
+            n = n // chunk_bytes * chunk_bytes
+        rows.append((n, code[s.dtype], orc.shape_tag(list(s.shape))))
+        arrays.append(inputs.to_numpy_bytes(views[0][t].view(-1).view(__import__("torch").uint8)[:n]))
+        picked.append(t)
+        total += n
+    return orc.make_tensor_table(rows), arrays, picked, total
+
+
+def time_oracle(tt, arrays, chunk_bytes, nthreads):
+    import numpy as np
+    from oracle import scout_oracle as orc
+    n_chunks = len(orc.chunk_table(tt, chunk_bytes))
+    sigs = np.zeros((n_chunks, 1), dtype=orc.SIG_DTYPE)
+    t0 = time.perf_counter()
+    orc.sign_replica(tt, arrays, chunk_bytes, sigs, 0, nthreads)
+    orc.vote(np.repeat(sigs, 2, axis=1))      # the vote is part of the path (negligible)
+    return time.perf_counter() - t0, sigs
+
+
+def cpu_baseline(w, views, seconds):
+    """Oracle GB/s on this host, all cores, on a bounded sample."""
+    cores = os.cpu_count() or 1
+    tt, arrays, picked, total = oracle_sample(w, views, w.chunk_bytes, 8 << 20)
+    dt, _ = time_oracle(tt, arrays, w.chunk_bytes, 1)
+    rate1 = total / dt
+    budget = int(min(max(rate1 * cores * seconds * 0.6, 32 << 20), 16 << 30))
+    tt, arrays, picked, total = oracle_sample(w, views, w.chunk_bytes, budget)
+    dt, sigs = time_oracle(tt, arrays, w.chunk_bytes, cores)
+    return {"value": total / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "single_thread_value": rate1 / 1e9,
+            "sample": f"leading whole chunks of replica 0: {total} bytes of {len(picked)} tensors, "
+                      f"{cores} threads over chunks, {dt:.1f} s"}, (tt, picked, sigs)
+
+
+def run_reference(args):
+    """The CPU oracle as the reference arm: same config, metric and unit; every
+    step signs and votes a bounded sample of the workload on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+    from paper_2608_11034_b200 import inputs
+    from oracle import scout_oracle as orc
+    orc.build()
+    w = inputs.workload(args.config, "default", args.scale)
+    cores = os.cpu_count() or 1
+    # generate only what is sampled: shrink each tensor to its leading chunks
+    budget = 192 << 20
+    per_tensor = max(w.chunk_bytes, budget // len(w.specs) // w.chunk_bytes * w.chunk_bytes)
+    specs, total = [], 0
+    for s in w.specs:
+        if total >= budget:
+            break
+        es = inputs.DTYPE_BYTES[s.dtype]
+        n = min(s.nbytes, per_tensor)
+        specs.append(inputs.TensorSpec(s.name, (n // es,), s.dtype, s.dist, s.std))
+        total += n
+    sw = inputs.Workload(w.name, w.config, "sample", w.R, w.chunk_bytes, specs, w.seed)
+    _, views0 = inputs.generate_replica0(sw, "cpu")
+    views = [views0]
+    tt, arrays, picked, total = oracle_sample(sw, views, sw.chunk_bytes, budget)
+    times = []
+    for i in range(args.warmup + args.steps):
+        dt, _ = time_oracle(tt, arrays, sw.chunk_bytes, cores)
+        if i >= args.warmup:
+            times.append(dt)
+    t = sum(times)
+    value = total * len(times) / t / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64+f64",
+        "data": "synthetic",
+        "config": {"workload": w.name, "R": w.R, "chunk_bytes": w.chunk_bytes,
+                   "sample_bytes_per_step": total},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"one replica's leading chunks, {total} bytes per step, {cores} threads"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------ the CUDA arm
+
+def expected_pairs(w, plan_handle, binding, inputs):
+    """(chunk, replica) pairs the fault patches must produce, from chunk geometry."""
+    import bisect
+    C = binding.scout_plan_num_chunks(plan_handle)
+    # chunk ids of a tensor are consecutive; find each tensor's first chunk
+    first, c = {}, 0
+    for t, s in enumerate(w.specs):
+        first[t] = c
+        c += (s.nbytes + w.chunk_bytes - 1) // w.chunk_bytes
+    assert c == C
+    pairs = set()
+    for p in w.patches:
+        es = inputs.DTYPE_BYTES[w.specs[p.tensor].dtype]
+        pairs.add((first[p.tensor] + (p.element * es) // w.chunk_bytes, p.replica))
+    return sorted(pairs)
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2608_11034_b200 import binding, inputs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the product path has no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    w = inputs.workload(args.config, "default", args.scale)
+    w.seed += 4096 * rank                    # every rank scans its own replica set
+    flats, views = inputs.generate(w, "cuda")
+    total_bytes = w.R * w.bytes_per_replica
+    small = total_bytes < (1 << 30)          # working set may sit in L2: flush between steps
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda") if small else None
+
+    plan = binding.Plan(w.R, binding.make_tensor_table(w.specs), w.chunk_bytes)
+    if args.tile_bytes:
+        binding.scout_plan_set(plan.handle, "tile_bytes", args.tile_bytes)
+    if args.variant is not None:
+        binding.scout_plan_set(plan.handle, "variant", args.variant)
+    binding.scout_plan_set(plan.handle, "timing", 1)
+    plan.bind(views)
+    use_certify = args.config == 4
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def step():
+        if use_certify:
+            return plan.certify()
+        plan.sign_and_vote()
+        return None
+
+    for _ in range(max(args.warmup, 0)):
+        step()
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+          for _ in range(args.steps)]
+    scan_ns = []
+    barrier()
+    torch.cuda.synchronize()
+    for i in range(args.steps):
+        if flush is not None:
+            flush.fill_(i & 255)
+        ev[i][0].record()
+        last = step()
+        ev[i][1].record()
+        if use_certify or small:
+            torch.cuda.synchronize()
+            scan_ns.append(binding.scout_plan_get(plan.handle, "last_sign_ns"))
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    if not scan_ns:
+        scan_ns.append(binding.scout_plan_get(plan.handle, "last_sign_ns"))
+    ms = sum(a.elapsed_time(b) for a, b in ev)
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+
+    # the last timed step must have produced the right answer
+    want = expected_pairs(w, plan.handle, binding, inputs)
+    if use_certify:
+        got = last["outliers"]
+        verdict = last["report"]["verdict"]
+    else:
+        res = plan.fetch()
+        got = res["outliers"]
+        verdict = None
+    verified = got == want
+    if not verified:
+        raise SystemExit(f"wrong result: outliers {got[:8]} expected {want[:8]}")
+
+    value = world * total_bytes * args.steps / (ms * 1e-3) / 1e9
+    peak, peak_kind = measured_peak()
+    scan_s = (sum(scan_ns) / len(scan_ns)) * 1e-9
+    achieved = total_bytes / scan_s / 1e9
+    C = plan.C
+    roofline = {
+        "bound": "hbm", "kernel": "sign_tiles", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "frac": achieved / peak, "peak_kind": peak_kind,
+        "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+        "algorithmic_bytes_per_launch": total_bytes,
+        "avg_launch_ms": scan_s * 1e3, "launches_timed": len(scan_ns),
+        "traffic": (SCAN_TRAFFIC_RATIO * total_bytes) if SCAN_TRAFFIC_RATIO else None,
+    }
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u64+f64", "data": "synthetic",
+        "config": {"workload": w.name, "R": w.R, "tensors": len(w.specs), "chunks": C,
+                   "chunk_bytes": w.chunk_bytes, "bytes_per_step_per_gpu": total_bytes,
+                   "call": "scout_certify" if use_certify else "scout_sign_chunks+scout_consensus_vote",
+                   "tile_bytes": binding.scout_plan_get(plan.handle, "tile_bytes"),
+                   "variant": binding.scout_plan_get(plan.handle, "variant"),
+                   "l2": "512 MiB written between steps" if small else "inputs far larger than L2, no flush",
+                   "parallelism": f"{world} independent replica sets" if world > 1 else "single GPU"},
+        "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
+        "frac_of_measured_copy": value / world / peak,
+        "verified": verified, "verdict": verdict,
+        "gpu_launches": 4 * args.steps if use_certify else 3 * args.steps,
+        "clocks": clocks, "roofline": roofline,
+    }
+
+    # ---- end to end: replicas in pinned host memory, copies inside the timed region
+    if not args.no_e2e and rank == 0 and world == 1:
+        try:
+            bad = sorted({p.replica for p in w.patches})
+            base = torch.empty(flats[0].numel(), dtype=torch.uint8, pin_memory=True)
+            clean = next(r for r in range(w.R) if r not in bad)
+            base.copy_(flats[clean])
+            host = {r: base for r in range(w.R) if r not in bad}
+            for r in bad:
+                h = torch.empty(flats[0].numel(), dtype=torch.uint8, pin_memory=True)
+                h.copy_(flats[r])
+                host[r] = h
+            hviews = [inputs.tensor_views(host[r], w.specs) for r in range(w.R)]
+            hptrs = [v.data_ptr() for rep in hviews for v in rep]
+            binding.scout_certify_host(plan.handle, hptrs)          # warm-up (allocates staging)
+            t0 = time.perf_counter()
+            for _ in range(args.e2e_steps):
+                rep = binding.scout_certify_host(plan.handle, hptrs)
+            dt = time.perf_counter() - t0
+            assert rep["outliers"] == want
+            line["e2e"] = {"value": total_bytes * args.e2e_steps / dt / 1e9, "unit": UNIT,
+                           "h2d_bytes_per_step": total_bytes,
+                           "d2h_bytes_per_step": 576 + 16 * len(want),
+                           "steps": args.e2e_steps, "call": "scout_certify_host",
+                           "host_memory": f"pinned; {len(bad) + 1} distinct replica images "
+                                          f"(clean replicas share one host image)"}
+            del base, host, hviews
+        except Exception as e:                                       # noqa: BLE001
+            line["e2e"] = {"value": None, "unit": UNIT, "error": repr(e)[:200]}
+    else:
+        line["e2e"] = {"value": None, "unit": UNIT, "note": "measured on rank 0 at N=1 only"}
+
+    # ---- CPU oracle on a bounded sample, with a parity spot check against the CUDA records
+    if not args.no_cpu_baseline and rank == 0 and world == 1:
+        from oracle import scout_oracle as orc
+        orc.build()
+        cb, (tt, picked, osigs) = cpu_baseline(w, views, args.cpu_seconds)
+        plan.sign()                              # records into a torch-owned buffer
+        torch.cuda.synchronize()
+        all_sigs = plan.d_sigs.cpu().numpy().view(binding.SIG_DTYPE).reshape(C, w.R)
+        first, c = {}, 0
+        for t, s in enumerate(w.specs):
+            first[t] = c
+            c += (s.nbytes + w.chunk_bytes - 1) // w.chunk_bytes
+        oc, ok = 0, True
+        for i, t in enumerate(picked):
+            n_ch = (int(tt[i]["nbytes"]) + w.chunk_bytes - 1) // w.chunk_bytes
+            for k in range(n_ch):
+                g, o = all_sigs[first[t] + k, 0], osigs[oc, 0]
+                ok &= int(g["hash"]) == int(o["hash"]) and g["nan_count"] == o["nan_count"]
+                ok &= abs(g["sumsq"] - o["sumsq"]) <= 1e-12 * abs(o["sumsq"])
+                oc += 1
+        cb["parity_spot_check"] = {"chunks": oc, "ok": bool(ok)}
+        line["cpu_baseline"] = cb
+        if not ok:
+            raise SystemExit("CUDA records disagree with the oracle on the sampled chunks")
+    else:
+        line["cpu_baseline"] = None
+
+    plan.close()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

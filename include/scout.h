@@ -187,10 +187,17 @@ SCOUT_API int scout_certify_host(scout_plan_t *plan, const void *const *h_ptrs /
 /* Shape tag for scout_tensor_t.meta_tag: a 64-bit digest of (ndim, dims). */
 SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/);
 
-/* Tuning knobs of a plan (optional; call before the first scout_sign_chunks).
- * key "tile_bytes": bytes per work item, a power of two in [2048, 65536];
- * key "variant": 0 = direct vector loads, 1 = bulk-async staging through
- * shared memory.  Results do not depend on either except for the rounding
+/* Knobs of a plan (optional).
+ *   set "tile_bytes"  bytes per work item, a power of two in [2048, 65536]
+ *   set "variant"     0 = direct vector loads, 1 = bulk-async staging through
+ *                     shared memory
+ *   set "grid"        CTAs of the scan kernel
+ *   set "timing"      1: record CUDA events around the scan kernel on the
+ *                     caller's stream
+ *   get "last_sign_ns" device time of the most recent scan kernel (needs
+ *                     "timing" and a synchronised stream)
+ *   get "n_tiles", "scratch_bytes", and every settable key
+ * Results do not depend on tile_bytes, variant or grid except for the rounding
  * order of the floating-point sums. */
 SCOUT_API int scout_plan_set(scout_plan_t *plan, const char *key, int64_t value);
 SCOUT_API int scout_plan_get(const scout_plan_t *plan, const char *key, int64_t *value);

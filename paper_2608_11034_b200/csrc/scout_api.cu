@@ -66,6 +66,10 @@ struct scout_plan {
     uint64_t stage_bytes = 0;
     cudaStream_t s_copy = nullptr, s_comp = nullptr;
     cudaEvent_t ev_copied[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr};
+
+    // optional in-stream timing of the scan kernel (key "timing")
+    bool timing = false;
+    cudaEvent_t ev_t0 = nullptr, ev_t1 = nullptr;
 };
 
 namespace {
@@ -127,8 +131,10 @@ int sign_all(scout_plan *p, cudaStream_t stream, scout_sig_t *d_sigs) {
     l.recs = p->d_recs;
     l.variant = p->variant;
     l.grid = p->grid;
+    if (p->timing) SCOUT_CUDA(cudaEventRecord(p->ev_t0, stream));
     int rc = launch_sign_tiles(l, stream);
     if (rc) return rc;
+    if (p->timing) SCOUT_CUDA(cudaEventRecord(p->ev_t1, stream));
     return launch_finalize(p->d_chunks, p->chunks.size(), p->R, p->d_recs, p->tiles.size(),
                            p->tile_bytes / ROW_BYTES, d_sigs, stream);
 }
@@ -335,6 +341,8 @@ int scout_plan_destroy(scout_plan_t *p) {
     }
     if (p->s_copy) cudaStreamDestroy(p->s_copy);
     if (p->s_comp) cudaStreamDestroy(p->s_comp);
+    if (p->ev_t0) cudaEventDestroy(p->ev_t0);
+    if (p->ev_t1) cudaEventDestroy(p->ev_t1);
     (void)cudaGetLastError();
     delete p;
     return SCOUT_OK;
@@ -496,6 +504,14 @@ int scout_plan_set(scout_plan_t *p, const char *key, int64_t value) {
         p->variant = (int)value;
         return sign_grid_size(p->variant, p->device, &p->grid);
     }
+    if (!std::strcmp(key, "timing")) {
+        if (value && !p->ev_t0) {
+            SCOUT_CUDA(cudaEventCreate(&p->ev_t0));
+            SCOUT_CUDA(cudaEventCreate(&p->ev_t1));
+        }
+        p->timing = value != 0;
+        return SCOUT_OK;
+    }
     if (!std::strcmp(key, "grid")) {
         if (value < 1 || value > 65535) return SCOUT_ERR_INVALID;
         p->grid = (int)value;
@@ -510,6 +526,13 @@ int scout_plan_get(const scout_plan_t *p, const char *key, int64_t *value) {
     else if (!std::strcmp(key, "variant")) *value = p->variant;
     else if (!std::strcmp(key, "grid")) *value = p->grid;
     else if (!std::strcmp(key, "n_tiles")) *value = (int64_t)p->tiles.size();
+    else if (!std::strcmp(key, "last_sign_ns")) {
+        // device time of the most recent scan kernel; the stream must have been synchronised
+        if (!p->timing || !p->ev_t0) return SCOUT_ERR_INVALID;
+        float ms = 0.f;
+        SCOUT_CUDA(cudaEventElapsedTime(&ms, p->ev_t0, p->ev_t1));
+        *value = (int64_t)((double)ms * 1e6);
+    }
     else if (!std::strcmp(key, "scratch_bytes")) *value = (int64_t)(p->tiles.size() * p->R * sizeof(TileRec));
     else return SCOUT_ERR_INVALID;
     return SCOUT_OK;
