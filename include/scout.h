@@ -184,6 +184,37 @@ SCOUT_API int scout_certify_host(scout_plan_t *plan, const void *const *h_ptrs /
                        scout_report_t *report /*host*/, scout_outlier_t *h_outliers,
                        uint64_t outlier_cap, uint64_t *h_undecided, uint64_t undecided_cap);
 
+/* ---- signing without allocating ---------------------------------------------
+ * (The paper has no counterpart: this entry point exists for deployment.)
+ * For callers that must not allocate device memory while they run, for example
+ * a check placed inside a training step whose framework already holds nearly
+ * all of HBM in its own allocator (a cudaMalloc there can fail, and it stalls
+ * the device), or a handler running right after an out-of-memory error.
+ * No plan is needed and nothing is allocated or freed, on the device or through
+ * any library: the per-tile partial records go to a fixed 2 MiB array inside
+ * the library's device image (every GPU that loads the library holds it until
+ * the process exits).
+ *   R             replicas, 2..64
+ *   replica_ptrs  host array of R device addresses, 16-byte aligned; replica r
+ *                 is ONE contiguous tensor of `nbytes` bytes at replica_ptrs[r]
+ *   nbytes, dtype, meta_tag, chunk_bytes   as in scout_tensor_t / scout_plan_create
+ *   d_sigs        device, caller-allocated, [C][R] with C = ceil(nbytes / chunk_bytes);
+ *                 same records as scout_sign_chunks for a one-tensor plan
+ *                 (hashes and counts identical; the fp64 sums may differ in the
+ *                 last bits because the tile size may differ)
+ * Limit: R * (number of 64 KiB tiles) <= 65536 records, i.e. about 4 GiB of
+ * replica data per call; more returns SCOUT_ERR_UNSUPPORTED and launches
+ * nothing.  The first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress, with that device current); make that first call
+ * before any stream capture.  All calls share the one array and every call
+ * overwrites the records it reads, so nothing needs clearing between calls,
+ * but two calls whose kernels overlap on the GPU (different streams, or several
+ * host threads) race on it: serialise them.  Asynchronous on `stream`. */
+SCOUT_API int scout_sign_chunks_noalloc(uint32_t R, const void *const *replica_ptrs /*host*/,
+                                        uint64_t nbytes, uint32_t dtype, uint64_t meta_tag,
+                                        uint64_t chunk_bytes, scout_sig_t *d_sigs /*device*/,
+                                        void *stream);
+
 /* Shape tag for scout_tensor_t.meta_tag: a 64-bit digest of (ndim, dims). */
 SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/);
 

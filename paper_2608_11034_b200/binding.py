@@ -71,6 +71,7 @@ def lib():
             "scout_plan_replica_bad_counts": (C.c_int, [vp, vp]),
             "scout_rollup_tensors": (C.c_int, [vp, vp, vp, vp]),
             "scout_certify_host": (C.c_int, [vp, vp, vp, vp, u64, vp, u64]),
+            "scout_sign_chunks_noalloc": (C.c_int, [u32, vp, u64, u32, u64, u64, vp, vp]),
             "scout_shape_tag": (u64, [u32, vp]),
             "scout_plan_set": (C.c_int, [vp, C.c_char_p, i64]),
             "scout_plan_get": (C.c_int, [vp, C.c_char_p, C.POINTER(i64)]),
@@ -193,6 +194,15 @@ def scout_plan_replica_bad_counts(plan: int, R: int) -> List[int]:
 
 def scout_rollup_tensors(plan: int, d_sigs: int, d_tensor_sigs: int, stream: int) -> None:
     _check(lib().scout_rollup_tensors(plan, d_sigs, d_tensor_sigs, stream), "scout_rollup_tensors")
+
+
+def scout_sign_chunks_noalloc(R: int, replica_ptrs: Sequence[int], nbytes: int, dtype: int,
+                              meta_tag: int, chunk_bytes: int, d_sigs: int, stream: int) -> None:
+    """Sign R one-tensor replicas without allocating anything (see scout.h for
+    who needs this and for the size limit).  d_sigs: device [C][R] records."""
+    a = np.asarray(list(replica_ptrs), dtype=np.uint64)
+    _check(lib().scout_sign_chunks_noalloc(R, a.ctypes.data, nbytes, dtype, meta_tag, chunk_bytes,
+                                           d_sigs, stream), "scout_sign_chunks_noalloc")
 
 
 def scout_version() -> int:
