@@ -35,9 +35,11 @@ METRIC = "replica GB/s scanned (sign+vote)"
 UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes per algorithmic byte of the scan kernel, from the ncu capture
-# summarised in profiles/ (None until a capture exists)
-SCAN_TRAFFIC_RATIO = None
+# DRAM bytes (read + write) per algorithmic byte of the scan kernel, from the ncu
+# captures summarised under profiles/: 1.8007 GB read + 0.026 GB written for
+# 1.8000 GB scanned (fp32), 1.1407 + 0.016 for 1.1401 GB (bf16).  Traffic grows
+# in proportion to the bytes scanned, so a full-size launch is scaled by this.
+SCAN_TRAFFIC_RATIO = 1.0148
 
 
 def measured_peak():
@@ -51,7 +53,7 @@ def measured_peak():
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=4, choices=[1, 2, 3, 4, 5])

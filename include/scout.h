@@ -220,13 +220,17 @@ SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/)
 
 /* Knobs of a plan (optional).
  *   set "tile_bytes"  bytes per work item, a power of two in [2048, 65536]
- *   set "variant"     0 = direct vector loads, 1 = bulk-async staging through
- *                     shared memory
+ *   set "variant"     scan kernel: 0 = direct 16-byte loads; 1 = the same with the
+ *                     next rows prefetched into registers; 2 = bulk-async copies
+ *                     (cp.async.bulk + mbarrier) through a per-warp ring in
+ *                     shared memory; 3 = read-only probe (measures the memory
+ *                     system only: the records it leaves are NOT signatures)
  *   set "grid"        CTAs of the scan kernel
  *   set "timing"      1: record CUDA events around the scan kernel on the
  *                     caller's stream
  *   get "last_sign_ns" device time of the most recent scan kernel (needs
  *                     "timing" and a synchronised stream)
+ *   get "device_error" 1 if a kernel's bounded wait ever gave up (synchronises)
  *   get "n_tiles", "scratch_bytes", and every settable key
  * Results do not depend on tile_bytes, variant or grid except for the rounding
  * order of the floating-point sums. */

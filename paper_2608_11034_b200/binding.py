@@ -16,7 +16,8 @@ from typing import List, Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libscout_b200.so")
+# SCOUT_LIB selects another build of the same library (e.g. other compile-time settings)
+LIB_PATH = os.environ.get("SCOUT_LIB") or os.path.join(_HERE, "libscout_b200.so")
 
 OK, ERR_INVALID, ERR_ALIGN, ERR_UNSUPPORTED, ERR_CUDA, ERR_NOMEM, ERR_TRUNCATED = 0, -1, -2, -3, -4, -5, -6
 DT_U8, DT_F32, DT_BF16, DT_I64, DT_F16, DT_F64, DT_I32 = range(7)

@@ -32,16 +32,19 @@ def is_stale() -> bool:
     return (not os.path.exists(LIB)) or os.path.getmtime(LIB) < max(os.path.getmtime(d) for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, out: str = LIB, defines=()) -> str:
+    """Compile the library.  ``out``/``defines`` build an alternative copy with
+    other -D settings (select it at run time with the SCOUT_LIB variable)."""
     srcs, _ = sources()
-    if not force and not is_stale():
+    if out == LIB and not force and not is_stale():
         return LIB
-    tmp = LIB + ".tmp%d" % os.getpid()
+    tmp = out + ".tmp%d" % os.getpid()
     cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
+          ["-D" + d for d in defines] + \
           ["-I", os.path.join(ROOT, "include"), "-I", CSRC, "-shared", "-o", tmp] + srcs
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, out)
+    return out
 
 
 if __name__ == "__main__":

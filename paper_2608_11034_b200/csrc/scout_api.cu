@@ -51,6 +51,7 @@ struct scout_plan {
     uint64_t *d_tensor_chunk0 = nullptr;
     const uint8_t **d_ptrs = nullptr;
     TileRec *d_recs = nullptr;
+    uint32_t *d_error = nullptr;  // set by a kernel whose bounded wait gave up
 
     // certify-owned results
     scout_sig_t *d_sigs = nullptr;
@@ -129,6 +130,7 @@ int sign_all(scout_plan *p, cudaStream_t stream, scout_sig_t *d_sigs) {
     l.stage = nullptr;
     l.slice_begin = 0;
     l.recs = p->d_recs;
+    l.error = p->d_error;
     l.variant = p->variant;
     l.grid = p->grid;
     if (p->timing) SCOUT_CUDA(cudaEventRecord(p->ev_t0, stream));
@@ -204,6 +206,13 @@ int vote_and_report(scout_plan *p, cudaStream_t stream, scout_report_t *report,
     report->verdict = o.counts[3] ? SCOUT_UNDECIDED
                                   : (o.counts[2] ? SCOUT_VERDICT_ATTRIBUTED : SCOUT_CERTIFIED);
     p->have_results = true;
+    uint32_t dev_err = 0;
+    SCOUT_CUDA(cudaMemcpyAsync(&dev_err, p->d_error, sizeof(dev_err), cudaMemcpyDeviceToHost, stream));
+    SCOUT_CUDA(cudaStreamSynchronize(stream));
+    if (dev_err) {
+        set_cuda_error(cudaErrorUnknown, "scan kernel: a bounded wait for a bulk copy gave up");
+        return SCOUT_ERR_CUDA;
+    }
     return (o.counts[4] > outlier_cap || o.counts[5] > undecided_cap) ? SCOUT_ERR_TRUNCATED : SCOUT_OK;
 }
 
@@ -272,8 +281,13 @@ int scout_plan_create(uint32_t R, uint64_t T, const scout_tensor_t *tensors, uin
         if ((rc = sign_grid_size(p->variant, p->device, &p->grid))) break;
         if ((rc = upload_tables(p))) break;
         if (cudaMalloc(&p->d_tensor_chunk0, (T + 1) * sizeof(uint64_t)) != cudaSuccess ||
-            cudaMalloc(&p->d_ptrs, (size_t)R * T * sizeof(void *)) != cudaSuccess) {
+            cudaMalloc(&p->d_ptrs, (size_t)R * T * sizeof(void *)) != cudaSuccess ||
+            cudaMalloc(&p->d_error, sizeof(uint32_t)) != cudaSuccess) {
             rc = SCOUT_ERR_NOMEM;
+            break;
+        }
+        if (cudaMemset(p->d_error, 0, sizeof(uint32_t)) != cudaSuccess) {
+            rc = SCOUT_ERR_CUDA;
             break;
         }
         if (cudaMemcpy(p->d_tensor_chunk0, p->tensor_chunk0.data(), (T + 1) * sizeof(uint64_t),
@@ -326,6 +340,7 @@ int scout_plan_destroy(scout_plan_t *p) {
     cudaFree(p->d_tensor_chunk0);
     cudaFree((void *)p->d_ptrs);
     cudaFree(p->d_recs);
+    cudaFree(p->d_error);
     cudaFree(p->d_sigs);
     cudaFree(p->d_status);
     cudaFree(p->d_bitmap);
@@ -433,7 +448,8 @@ int scout_certify_host(scout_plan_t *p, const void *const *h_ptrs, scout_report_
             l.stage = p->d_stage[buf];
             l.slice_begin = a;
             l.recs = p->d_recs;
-            l.variant = p->variant;
+            l.error = p->d_error;
+            l.variant = p->variant == 3 ? 0 : p->variant;
             l.grid = p->grid;
             if ((rc = launch_sign_tiles(l, p->s_comp))) return rc;
             SCOUT_CUDA(cudaEventRecord(p->ev_done[buf], p->s_comp));
@@ -500,7 +516,7 @@ int scout_plan_set(scout_plan_t *p, const char *key, int64_t value) {
         return upload_tables(p);
     }
     if (!std::strcmp(key, "variant")) {
-        if (value < 0 || value > 1) return SCOUT_ERR_INVALID;
+        if (value < 0 || value > 3) return SCOUT_ERR_INVALID;
         p->variant = (int)value;
         return sign_grid_size(p->variant, p->device, &p->grid);
     }
@@ -532,6 +548,11 @@ int scout_plan_get(const scout_plan_t *p, const char *key, int64_t *value) {
         float ms = 0.f;
         SCOUT_CUDA(cudaEventElapsedTime(&ms, p->ev_t0, p->ev_t1));
         *value = (int64_t)((double)ms * 1e6);
+    }
+    else if (!std::strcmp(key, "device_error")) {
+        uint32_t e = 0;
+        SCOUT_CUDA(cudaMemcpy(&e, p->d_error, sizeof(e), cudaMemcpyDeviceToHost));
+        *value = e;
     }
     else if (!std::strcmp(key, "scratch_bytes")) *value = (int64_t)(p->tiles.size() * p->R * sizeof(TileRec));
     else return SCOUT_ERR_INVALID;

@@ -122,7 +122,8 @@ struct SignLaunch {
     const uint8_t *stage;         // staged mode: device image of packed bytes [slice_begin, ...)
     uint64_t slice_begin;         // packed offset held at stage[0]
     TileRec *recs;                // device [R][tiles_per_replica]
-    int variant;
+    uint32_t *error;              // device flag set when a bounded wait gave up (may be null)
+    int variant;                  // 0 direct, 1 direct + register prefetch, 2 bulk-async ring, 3 read probe
     int grid;                     // CTAs to launch
 };
 int launch_sign_tiles(const SignLaunch &a, cudaStream_t stream);

@@ -18,13 +18,31 @@
 // element, counts NaN/Inf and sums the finite ones only.
 #include <cuda_fp16.h>
 
+#include <type_traits>
+
 #include "scout_internal.h"
 
 namespace scout {
 namespace {
 
 constexpr int SIGN_THREADS = 256;
-constexpr int UNROLL = 4;
+#ifndef SCOUT_MINBLOCKS
+#define SCOUT_MINBLOCKS 4
+#endif
+#ifndef SCOUT_MINBLOCKS_PF
+#define SCOUT_MINBLOCKS_PF 3
+#endif
+#ifndef SCOUT_UNROLL
+#define SCOUT_UNROLL 8
+#endif
+constexpr int UNROLL = SCOUT_UNROLL;
+// bf16: how many of a word-quad's four high halves are widened by bit placement
+// instead of the conversion pipe (see stats_fast).
+#ifndef SCOUT_BF16_BITROUTE
+#define SCOUT_BF16_BITROUTE 2
+#endif
+
+constexpr int BF16_BITROUTE = SCOUT_BF16_BITROUTE;
 
 struct Acc {
     double s0, s1, q0, q1;
@@ -67,16 +85,57 @@ __device__ __forceinline__ void stats_fast(const uint4 &v, Acc &a) {
         acc2(a, (double)__uint_as_float(v.x), (double)__uint_as_float(v.y));
         acc2(a, (double)__uint_as_float(v.z), (double)__uint_as_float(v.w));
     } else if constexpr (DT == SCOUT_DT_BF16) {
+        // Two widening routes, mixed so that the conversion pipe (16 lanes/clk/SM)
+        // does not carry all eight elements of a vector.
+        //  (A) cvt.f64.bf16 straight from either half of the word; accumulators
+        //      s0, q0 hold true values.
+        //  (B) bit placement, no conversion: the bf16 pattern dropped into the top
+        //      of a double's exponent/mantissa gives u = x * 2^-896 exactly for
+        //      every finite x (zeros and subnormals included); OR-ing 0x700 into
+        //      the exponent field gives v = x * 2^+896 for every NORMAL x (garbage
+        //      but finite for zeros and subnormals), so u*v = x^2 exactly for
+        //      normal x and for zero.  s1 sums u (rescaled once per tile), q1 sums
+        //      u*v.  A subnormal x contributes a wrong but tiny (< 2^-252) term to
+        //      q1; lanes with 0 < q1 < 2^-180 send the tile to the exact rescan, so
+        //      the error that can remain is below 2^-58 relative.
+        //      Inf/NaN give v = Inf/NaN: the usual "sum of squares not finite" flag.
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-            acc2(a, (double)__uint_as_float(w[i] << 16), (double)__uint_as_float(w[i] & 0xFFFF0000u));
+        for (int i = 0; i < 4; ++i) {
+            uint16_t l16, h16;
+            asm("mov.b32 {%0,%1}, %2;" : "=h"(l16), "=h"(h16) : "r"(w[i]));
+            double lo;
+            asm("cvt.f64.bf16 %0, %1;" : "=d"(lo) : "h"(l16));
+            a.s0 += lo;
+            a.q0 = fma(lo, lo, a.q0);
+            if (i < BF16_BITROUTE) {
+                const uint32_t uh = (uint32_t)((int)w[i] >> 3) & 0x8FFFE000u;
+                const double u = __hiloint2double((int)uh, 0);
+                const double x2 = __hiloint2double((int)(uh | 0x70000000u), 0);
+                a.s1 += u;
+                a.q1 = fma(u, x2, a.q1);
+            } else {
+                double hi;
+                asm("cvt.f64.bf16 %0, %1;" : "=d"(hi) : "h"(h16));
+                if (BF16_BITROUTE > 0) {
+                    a.s0 += hi;
+                    a.q0 = fma(hi, hi, a.q0);
+                } else {
+                    a.s1 += hi;
+                    a.q1 = fma(hi, hi, a.q1);
+                }
+            }
+        }
     } else if constexpr (DT == SCOUT_DT_F16) {
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
-            acc2(a, (double)f.x, (double)f.y);
+            uint16_t l16, h16;
+            double lo, hi;
+            asm("mov.b32 {%0,%1}, %2;" : "=h"(l16), "=h"(h16) : "r"(w[i]));
+            asm("cvt.f64.f16 %0, %1;" : "=d"(lo) : "h"(l16));
+            asm("cvt.f64.f16 %0, %1;" : "=d"(hi) : "h"(h16));
+            acc2(a, lo, hi);
         }
     } else if constexpr (DT == SCOUT_DT_F64) {
         acc2(a, __hiloint2double((int)v.y, (int)v.x), __hiloint2double((int)v.w, (int)v.z));
@@ -91,7 +150,11 @@ __device__ __forceinline__ void stats_fast(const uint4 &v, Acc &a) {
 
 template <int DT>
 __device__ __forceinline__ bool may_hold_nonfinite(const Acc &a) {
-    if constexpr (DT == SCOUT_DT_F32 || DT == SCOUT_DT_BF16 || DT == SCOUT_DT_F16) {
+    if constexpr (DT == SCOUT_DT_BF16) {
+        // non-finite element, or a subnormal one on the bit-placement route
+        return !(a.q0 + a.q1 < 1.157920892373162e77) ||                    // 2^256
+               (BF16_BITROUTE > 0 && a.q1 > 0.0 && a.q1 < 6.525304467998525e-55);  // 2^-180
+    } else if constexpr (DT == SCOUT_DT_F32 || DT == SCOUT_DT_F16) {
         return !(a.q0 + a.q1 < 1.157920892373162e77);  // 2^256
     } else if constexpr (DT == SCOUT_DT_F64) {
         return !(a.q0 + a.q1 < __longlong_as_double(0x7FF0000000000000ll));
@@ -171,66 +234,153 @@ __device__ __noinline__ void rescan_classifying(const uint8_t *tile, uint32_t nb
     inf_count = a.inf_count;
 }
 
+// h <- h * P + (m0 w0 + m1 w1 + m2 w2 + m3 w3) mod 2^64.
+#ifndef SCOUT_FOLD_IMPL
+#define SCOUT_FOLD_IMPL 1
+#endif
 __device__ __forceinline__ void fold_row(uint64_t &h, const uint4 &v, const uint32_t (&m)[4]) {
+#if SCOUT_FOLD_IMPL == 0
     uint64_t s = (uint64_t)m[0] * v.x;
     s += (uint64_t)m[1] * v.y;
     s += (uint64_t)m[2] * v.z;
     s += (uint64_t)m[3] * v.w;
     h = h * HASH_P + s;
+#elif SCOUT_FOLD_IMPL == 1
+    uint64_t t = h * HASH_P;
+    t += (uint64_t)m[0] * v.x;
+    t += (uint64_t)m[1] * v.y;
+    t += (uint64_t)m[2] * v.z;
+    t += (uint64_t)m[3] * v.w;
+    h = t;
+#elif SCOUT_FOLD_IMPL == 2
+    uint64_t t = h * HASH_P;
+    asm("mad.wide.u32 %0, %1, %2, %0;" : "+l"(t) : "r"(m[0]), "r"(v.x));
+    asm("mad.wide.u32 %0, %1, %2, %0;" : "+l"(t) : "r"(m[1]), "r"(v.y));
+    asm("mad.wide.u32 %0, %1, %2, %0;" : "+l"(t) : "r"(m[2]), "r"(v.z));
+    asm("mad.wide.u32 %0, %1, %2, %0;" : "+l"(t) : "r"(m[3]), "r"(v.w));
+    h = t;
+#else
+    // explicit 32-bit pieces: low/high words of h*P by hand, products by mad.wide
+    const uint32_t hl = (uint32_t)h, hh = (uint32_t)(h >> 32);
+    const uint32_t pl = (uint32_t)HASH_P, ph = (uint32_t)(HASH_P >> 32);
+    uint64_t t = (uint64_t)hl * pl;
+    uint32_t thi = (uint32_t)(t >> 32) + hl * ph + hh * pl;
+    t = ((uint64_t)thi << 32) | (uint32_t)t;
+    uint64_t sa = (uint64_t)m[0] * v.x + (uint64_t)m[1] * v.y;
+    uint64_t sb = (uint64_t)m[2] * v.z + (uint64_t)m[3] * v.w;
+    h = t + sa + sb;
+#endif
 }
 
-// One warp scans one tile with direct 16-byte loads.
+// Per-lane state of one tile's scan: the lane's four slot multipliers, its share
+// of the hash recurrence, and its fp64 accumulators.  Rows may be fed from
+// registers (direct loads) or from shared memory (bulk-async ring); the
+// arithmetic is the same.
+template <int DT>
+struct TileScan {
+    uint32_t m[4];
+    uint64_t h;
+    Acc a;
+
+    __device__ __forceinline__ void begin(uint32_t lane) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) m[j] = ((4u * lane + j + 1u) * HASH_G32) | 1u;
+        h = 0;
+        a = Acc{0.0, 0.0, 0.0, 0.0};
+    }
+    __device__ __forceinline__ void row(const uint4 &v) {
+        fold_row(h, v, m);
+        stats_fast<DT>(v, a);
+    }
+    // Ragged last row of a chunk (missing words are zero), warp reduction, and the
+    // classifying rescan if the tile may hold a non-finite element.
+    __device__ __forceinline__ void finish(const uint8_t *tile, uint32_t nbytes, uint32_t lane,
+                                           TileRec &out) {
+        if (nbytes % ROW_BYTES) {
+            uint4 v = ld_masked16(tile, (nbytes / ROW_BYTES) * ROW_BYTES + 16u * lane, nbytes);
+            row(v);
+        }
+        double s, q = a.q0 + a.q1;
+        if constexpr (DT == SCOUT_DT_BF16 && BF16_BITROUTE > 0)
+            s = fma(a.s1, 0x1p896, a.s0);  // s1 holds x * 2^-896: exact power-of-two rescale
+        else
+            s = a.s0 + a.s1;
+        const bool suspect = __any_sync(0xFFFFFFFFu, may_hold_nonfinite<DT>(a));
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) {
+            h += __shfl_xor_sync(0xFFFFFFFFu, h, d);
+            s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
+            q += __shfl_xor_sync(0xFFFFFFFFu, q, d);
+        }
+        uint32_t nan_count = 0, inf_count = 0;
+        if constexpr (DT == SCOUT_DT_F32 || DT == SCOUT_DT_BF16 || DT == SCOUT_DT_F16 ||
+                      DT == SCOUT_DT_F64) {
+            if (suspect) rescan_classifying<DT>(tile, nbytes, lane, s, q, nan_count, inf_count);
+        }
+        out.h = h;
+        out.sum = s;
+        out.sumsq = q;
+        out.nan_count = nan_count;
+        out.inf_count = inf_count;
+    }
+};
+
+// Front end 0: one warp scans one tile with direct 16-byte loads, UNROLL rows in
+// flight, no overlap of a warp's own loads with its own arithmetic.
 template <int DT>
 __device__ __forceinline__ void scan_tile(const uint8_t *tile, uint32_t nbytes, uint32_t lane,
                                           TileRec &out) {
-    uint32_t m[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) m[j] = ((4u * lane + j + 1u) * HASH_G32) | 1u;
-
+    TileScan<DT> st;
+    st.begin(lane);
     const uint32_t full = nbytes / ROW_BYTES;
     const uint8_t *p = tile + 16u * lane;
-    uint64_t h = 0;
-    Acc a = {0.0, 0.0, 0.0, 0.0};
-    uint32_t row = 0;
-    for (; row + UNROLL <= full; row += UNROLL) {
+#pragma unroll 1
+    for (uint32_t b = full / UNROLL; b != 0; --b, p += UNROLL * ROW_BYTES) {
         uint4 v[UNROLL];
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u) v[u] = ld_stream16(p + (size_t)(row + u) * ROW_BYTES);
+        for (int u = 0; u < UNROLL; ++u) v[u] = ld_stream16(p + u * ROW_BYTES);
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-            fold_row(h, v[u], m);
-            stats_fast<DT>(v[u], a);
-        }
+        for (int u = 0; u < UNROLL; ++u) st.row(v[u]);
     }
-    for (; row < full; ++row) {
-        uint4 v = ld_stream16(p + (size_t)row * ROW_BYTES);
-        fold_row(h, v, m);
-        stats_fast<DT>(v, a);
-    }
-    if (nbytes % ROW_BYTES) {  // ragged last row of a chunk: missing words are zero
-        uint4 v = ld_masked16(tile, full * ROW_BYTES + 16u * lane, nbytes);
-        fold_row(h, v, m);
-        stats_fast<DT>(v, a);
-    }
+#pragma unroll 1
+    for (uint32_t b = full % UNROLL; b != 0; --b, p += ROW_BYTES) st.row(ld_stream16(p));
+    st.finish(tile, nbytes, lane, out);
+}
 
-    double s = a.s0 + a.s1, q = a.q0 + a.q1;
-    const bool suspect = __any_sync(0xFFFFFFFFu, may_hold_nonfinite<DT>(a));
+// Front end 1: rotating register pipeline.  PF_ROWS rows are always in flight:
+// as soon as a row has been folded its registers are reloaded with the row
+// PF_ROWS ahead, so a warp's loads overlap its own arithmetic.
+constexpr int PF_ROWS = 4;
+
+template <int DT>
+__device__ __forceinline__ void scan_tile_prefetch(const uint8_t *tile, uint32_t nbytes, uint32_t lane,
+                                                   TileRec &out) {
+    TileScan<DT> st;
+    st.begin(lane);
+    const uint32_t full = nbytes / ROW_BYTES;
+    const uint8_t *p = tile + 16u * lane;
+    const uint8_t *const end_full = p + (size_t)full * ROW_BYTES;
+    if (full >= PF_ROWS) {
+        // rows [p, p + PF_ROWS) are in registers; the loop reloads each register with
+        // the row PF_ROWS further on while there are at least PF_ROWS more rows
+        const uint8_t *const end_steady = p + (size_t)(full / PF_ROWS - 1) * (PF_ROWS * ROW_BYTES);
+        uint4 v[PF_ROWS];
 #pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) {
-        h += __shfl_xor_sync(0xFFFFFFFFu, h, d);
-        s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
-        q += __shfl_xor_sync(0xFFFFFFFFu, q, d);
+        for (int u = 0; u < PF_ROWS; ++u) v[u] = ld_stream16(p + u * ROW_BYTES);
+#pragma unroll 1
+        for (; p != end_steady; p += PF_ROWS * ROW_BYTES) {
+#pragma unroll
+            for (int u = 0; u < PF_ROWS; ++u) {
+                st.row(v[u]);
+                v[u] = ld_stream16(p + (PF_ROWS + u) * ROW_BYTES);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < PF_ROWS; ++u) st.row(v[u]);
+        p += PF_ROWS * ROW_BYTES;
     }
-    uint32_t nan_count = 0, inf_count = 0;
-    if constexpr (DT == SCOUT_DT_F32 || DT == SCOUT_DT_BF16 || DT == SCOUT_DT_F16 ||
-                  DT == SCOUT_DT_F64) {
-        if (suspect) rescan_classifying<DT>(tile, nbytes, lane, s, q, nan_count, inf_count);
-    }
-    out.h = h;
-    out.sum = s;
-    out.sumsq = q;
-    out.nan_count = nan_count;
-    out.inf_count = inf_count;
+    for (; p != end_full; p += ROW_BYTES) st.row(ld_stream16(p));
+    st.finish(tile, nbytes, lane, out);
 }
 
 struct SignArgs {
@@ -242,6 +392,7 @@ struct SignArgs {
     const uint8_t *stage;
     uint64_t slice_begin;
     TileRec *recs;
+    uint32_t *error;  // device flag: set if a bounded wait gave up
 };
 
 __device__ __forceinline__ void scan_dispatch(uint32_t dtype, const uint8_t *tile, uint32_t nbytes,
@@ -257,8 +408,34 @@ __device__ __forceinline__ void scan_dispatch(uint32_t dtype, const uint8_t *til
     }
 }
 
+__device__ __forceinline__ void scan_dispatch_prefetch(uint32_t dtype, const uint8_t *tile,
+                                                       uint32_t nbytes, uint32_t lane, TileRec &rec) {
+    switch (dtype) {
+        case SCOUT_DT_F32:  scan_tile_prefetch<SCOUT_DT_F32>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_BF16: scan_tile_prefetch<SCOUT_DT_BF16>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_I64:  scan_tile_prefetch<SCOUT_DT_I64>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_F16:  scan_tile_prefetch<SCOUT_DT_F16>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_F64:  scan_tile_prefetch<SCOUT_DT_F64>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_I32:  scan_tile_prefetch<SCOUT_DT_I32>(tile, nbytes, lane, rec); break;
+        default:            scan_tile_prefetch<SCOUT_DT_U8>(tile, nbytes, lane, rec); break;
+    }
+}
+
+__device__ __forceinline__ const uint8_t *tile_address(const SignArgs &a, const TileDesc &td, uint32_t r) {
+    return a.ptrs ? a.ptrs[(uint64_t)r * a.T + td.tensor] + td.off : a.stage + (td.poff - a.slice_begin);
+}
+
+__device__ __forceinline__ void store_record(TileRec *dst_rec, const TileRec &rec) {
+    uint4 *dst = reinterpret_cast<uint4 *>(dst_rec);
+    dst[0] = make_uint4((uint32_t)rec.h, (uint32_t)(rec.h >> 32), (uint32_t)__double2loint(rec.sum),
+                        (uint32_t)__double2hiint(rec.sum));
+    dst[1] = make_uint4((uint32_t)__double2loint(rec.sumsq), (uint32_t)__double2hiint(rec.sumsq),
+                        rec.nan_count, rec.inf_count);
+}
+
 // Persistent grid; every warp takes whole tiles, replica-major, round-robin.
-__global__ void __launch_bounds__(SIGN_THREADS) sign_tiles_direct(const SignArgs a) {
+template <int PREFETCH>
+__global__ void __launch_bounds__(SIGN_THREADS, PREFETCH ? SCOUT_MINBLOCKS_PF : SCOUT_MINBLOCKS) sign_tiles_direct(const SignArgs a) {
     const uint32_t lane = threadIdx.x & 31u;
     const uint64_t warp = (uint64_t)blockIdx.x * (SIGN_THREADS / 32) + (threadIdx.x >> 5);
     const uint64_t n_warps = (uint64_t)gridDim.x * (SIGN_THREADS / 32);
@@ -268,17 +445,227 @@ __global__ void __launch_bounds__(SIGN_THREADS) sign_tiles_direct(const SignArgs
         const uint64_t t = a.tile_begin + (item - (uint64_t)rr * a.n_tiles);
         const uint32_t r = a.replica_begin + rr;
         const TileDesc td = a.tiles[t];
-        const uint8_t *tile = a.ptrs ? a.ptrs[(uint64_t)r * a.T + td.tensor] + td.off
-                                     : a.stage + (td.poff - a.slice_begin);
+        const uint8_t *tile = tile_address(a, td, r);
         TileRec rec;
-        scan_dispatch(td.dtype, tile, td.nbytes, lane, rec);
-        if (lane == 0) {
-            uint4 *dst = reinterpret_cast<uint4 *>(&a.recs[(uint64_t)r * a.tiles_per_replica + t]);
-            dst[0] = make_uint4((uint32_t)rec.h, (uint32_t)(rec.h >> 32),
-                                (uint32_t)__double2loint(rec.sum), (uint32_t)__double2hiint(rec.sum));
-            dst[1] = make_uint4((uint32_t)__double2loint(rec.sumsq), (uint32_t)__double2hiint(rec.sumsq),
-                                rec.nan_count, rec.inf_count);
+        if (PREFETCH) scan_dispatch_prefetch(td.dtype, tile, td.nbytes, lane, rec);
+        else          scan_dispatch(td.dtype, tile, td.nbytes, lane, rec);
+        if (lane == 0) store_record(&a.recs[(uint64_t)r * a.tiles_per_replica + t], rec);
+    }
+}
+
+// ---- front end 2: bulk-async ring ----------------------------------------------
+// Every warp owns RING_STAGES pieces of RING_PIECE bytes in shared memory and one
+// mbarrier per piece.  Lane 0 asks the copy engine for whole rows
+// (cp.async.bulk global -> shared, completion counted in bytes on the piece's
+// mbarrier); the warp waits for a piece, folds its rows from shared memory, and
+// immediately asks for the piece RING_STAGES ahead, across tile boundaries, so
+// the bytes in flight do not depend on how long the arithmetic takes.  There is
+// no block-wide synchronisation: warps are independent.  Only whole rows go
+// through the ring; a chunk's ragged last row is read with plain loads.
+constexpr int RING_PIECE = 4096;  // 8 rows
+constexpr int RING_STAGES = 3;
+constexpr int RING_WARPS = SIGN_THREADS / 32;
+constexpr int RING_SMEM = RING_WARPS * RING_STAGES * RING_PIECE + RING_WARPS * RING_STAGES * 8;
+constexpr uint32_t RING_WAIT_LIMIT = 1u << 24;  // polls before a wait gives up
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+        "l"(src), "r"(bytes), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ uint4 lds16(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "r"(addr));
+    return v;
+}
+
+// The next piece the copy engine should fetch for this warp.
+struct PieceCursor {
+    uint64_t item;          // index into the warp's item sequence (global item id)
+    const uint8_t *base;    // tile address
+    uint32_t full_bytes;    // whole rows of the tile, in bytes
+    uint32_t offset;        // next byte of the tile to request
+    bool valid;
+};
+
+template <int DT>
+__device__ __forceinline__ void fold_piece(TileScan<DT> &st, uint32_t saddr, uint32_t rows) {
+    if (rows == RING_PIECE / ROW_BYTES) {
+#pragma unroll
+        for (int r = 0; r < RING_PIECE / (int)ROW_BYTES; ++r) st.row(lds16(saddr + r * ROW_BYTES));
+    } else {
+        for (uint32_t r = 0; r < rows; ++r) st.row(lds16(saddr + r * ROW_BYTES));
+    }
+}
+
+__global__ void __launch_bounds__(SIGN_THREADS, 2) sign_tiles_ring(const SignArgs a) {
+    extern __shared__ __align__(128) uint8_t ring_smem[];
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t wib = threadIdx.x >> 5;
+    const uint64_t warp = (uint64_t)blockIdx.x * RING_WARPS + wib;
+    const uint64_t n_warps = (uint64_t)gridDim.x * RING_WARPS;
+    const uint64_t n_items = a.n_tiles * a.n_replicas;
+    const uint32_t data0 = smem_u32(ring_smem) + wib * (RING_STAGES * RING_PIECE);
+    const uint32_t bar0 = smem_u32(ring_smem) + RING_WARPS * RING_STAGES * RING_PIECE + wib * (RING_STAGES * 8);
+
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < RING_STAGES; ++s) mbar_init(bar0 + 8 * s, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncwarp();
+
+    auto locate = [&](uint64_t item, TileDesc &td, uint32_t &r, uint64_t &t) {
+        const uint32_t rr = (uint32_t)(item / a.n_tiles);
+        t = a.tile_begin + (item - (uint64_t)rr * a.n_tiles);
+        r = a.replica_begin + rr;
+        td = a.tiles[t];
+    };
+    // move the cursor to the first item at or after `item` that has whole rows
+    auto seek = [&](PieceCursor &c, uint64_t item) {
+        c.valid = false;
+        for (; item < n_items; item += n_warps) {
+            TileDesc td;
+            uint32_t r;
+            uint64_t t;
+            locate(item, td, r, t);
+            const uint32_t fb = (td.nbytes / ROW_BYTES) * ROW_BYTES;
+            if (fb) {
+                c.item = item;
+                c.base = tile_address(a, td, r);
+                c.full_bytes = fb;
+                c.offset = 0;
+                c.valid = true;
+                return;
+            }
         }
+    };
+    uint32_t issued = 0;  // pieces requested so far; piece n lives in stage n % RING_STAGES
+    auto request = [&](PieceCursor &c) {
+        const uint32_t stage = issued % RING_STAGES;
+        const uint32_t bytes = min((uint32_t)RING_PIECE, c.full_bytes - c.offset);
+        if (lane == 0) {
+            mbar_expect_tx(bar0 + 8 * stage, bytes);
+            bulk_g2s(data0 + stage * RING_PIECE, c.base + c.offset, bytes, bar0 + 8 * stage);
+        }
+        ++issued;
+        c.offset += bytes;
+        if (c.offset >= c.full_bytes) seek(c, c.item + n_warps);
+    };
+
+    PieceCursor cur;
+    seek(cur, warp);
+    for (int s = 0; s < RING_STAGES && cur.valid; ++s) request(cur);
+
+    uint32_t consumed = 0;
+    bool gave_up = false;
+    for (uint64_t item = warp; item < n_items && !gave_up; item += n_warps) {
+        TileDesc td;
+        uint32_t r;
+        uint64_t t;
+        locate(item, td, r, t);
+        const uint8_t *tile = tile_address(a, td, r);
+        const uint32_t full_rows = td.nbytes / ROW_BYTES;
+        TileRec rec;
+        auto run = [&](auto tag) {
+            constexpr int DT = decltype(tag)::value;
+            TileScan<DT> st;
+            st.begin(lane);
+            for (uint32_t row0 = 0; row0 < full_rows; row0 += RING_PIECE / ROW_BYTES) {
+                const uint32_t stage = consumed % RING_STAGES;
+                const uint32_t parity = (consumed / RING_STAGES) & 1u;
+                uint32_t polls = 0;
+                while (!mbar_try_wait(bar0 + 8 * stage, parity)) {
+                    if (++polls > RING_WAIT_LIMIT) { gave_up = true; break; }
+                }
+                if (gave_up) break;
+                const uint32_t rows = min((uint32_t)(RING_PIECE / ROW_BYTES), full_rows - row0);
+                fold_piece<DT>(st, data0 + stage * RING_PIECE + 16u * lane, rows);
+                __syncwarp();  // every lane has read the piece before it is requested again
+                ++consumed;
+                if (cur.valid) request(cur);
+            }
+            if (!gave_up) st.finish(tile, td.nbytes, lane, rec);
+        };
+        switch (td.dtype) {
+            case SCOUT_DT_F32:  run(std::integral_constant<int, SCOUT_DT_F32>{}); break;
+            case SCOUT_DT_BF16: run(std::integral_constant<int, SCOUT_DT_BF16>{}); break;
+            case SCOUT_DT_I64:  run(std::integral_constant<int, SCOUT_DT_I64>{}); break;
+            case SCOUT_DT_F16:  run(std::integral_constant<int, SCOUT_DT_F16>{}); break;
+            case SCOUT_DT_F64:  run(std::integral_constant<int, SCOUT_DT_F64>{}); break;
+            case SCOUT_DT_I32:  run(std::integral_constant<int, SCOUT_DT_I32>{}); break;
+            default:            run(std::integral_constant<int, SCOUT_DT_U8>{}); break;
+        }
+        if (!gave_up && lane == 0) store_record(&a.recs[(uint64_t)r * a.tiles_per_replica + t], rec);
+    }
+    if (gave_up) {
+        // A copy never completed.  Report it, give the copies still in flight one more
+        // bounded chance to land (shared memory must not be released under them), return.
+        if (lane == 0 && a.error) atomicExch(a.error, 1u);
+        for (uint32_t n = consumed; n < issued; ++n) {
+            const uint32_t stage = n % RING_STAGES, parity = (n / RING_STAGES) & 1u;
+            uint32_t polls = 0;
+            while (!mbar_try_wait(bar0 + 8 * stage, parity) && ++polls <= RING_WAIT_LIMIT) {}
+        }
+    }
+}
+
+// Read-only probe: the same tiles and the same loads as the direct scan, with an
+// XOR as the only arithmetic.  It measures what the memory system delivers to
+// this access pattern (the ceiling the scan is compared with).
+__global__ void __launch_bounds__(SIGN_THREADS) read_probe(const SignArgs a) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint64_t warp = (uint64_t)blockIdx.x * (SIGN_THREADS / 32) + (threadIdx.x >> 5);
+    const uint64_t n_warps = (uint64_t)gridDim.x * (SIGN_THREADS / 32);
+    const uint64_t n_items = a.n_tiles * a.n_replicas;
+    for (uint64_t item = warp; item < n_items; item += n_warps) {
+        const uint32_t rr = (uint32_t)(item / a.n_tiles);
+        const uint64_t t = a.tile_begin + (item - (uint64_t)rr * a.n_tiles);
+        const uint32_t r = a.replica_begin + rr;
+        const TileDesc td = a.tiles[t];
+        const uint8_t *p = tile_address(a, td, r) + 16u * lane;
+        const uint32_t full = td.nbytes / ROW_BYTES;
+        uint4 x = make_uint4(0u, 0u, 0u, 0u);
+        uint32_t row = 0;
+        for (; row + 8 <= full; row += 8) {
+            uint4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = ld_stream16(p + (size_t)(row + u) * ROW_BYTES);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { x.x ^= v[u].x; x.y ^= v[u].y; x.z ^= v[u].z; x.w ^= v[u].w; }
+        }
+        for (; row < full; ++row) {
+            uint4 v = ld_stream16(p + (size_t)row * ROW_BYTES);
+            x.x ^= v.x; x.y ^= v.y; x.z ^= v.z; x.w ^= v.w;
+        }
+        uint32_t y = x.x ^ x.y ^ x.z ^ x.w;
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) y ^= __shfl_xor_sync(0xFFFFFFFFu, y, d);
+        if (lane == 0) a.recs[(uint64_t)r * a.tiles_per_replica + t].h = y;
     }
 }
 
@@ -355,8 +742,14 @@ __global__ void __launch_bounds__(FIN_THREADS) finalize_chunks(const ChunkDesc *
 int sign_grid_size(int variant, int device, int *grid) {
     int sms = 0, per_sm = 0;
     SCOUT_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
-    (void)variant;
-    SCOUT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sign_tiles_direct, SIGN_THREADS, 0));
+    if (variant == 2) {
+        SCOUT_CUDA(cudaFuncSetAttribute(sign_tiles_ring, cudaFuncAttributeMaxDynamicSharedMemorySize, RING_SMEM));
+        SCOUT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sign_tiles_ring, SIGN_THREADS, RING_SMEM));
+    } else if (variant == 1) {
+        SCOUT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sign_tiles_direct<1>, SIGN_THREADS, 0));
+    } else {
+        SCOUT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sign_tiles_direct<0>, SIGN_THREADS, 0));
+    }
     if (per_sm < 1) per_sm = 1;
     *grid = sms * per_sm;
     return SCOUT_OK;
@@ -376,11 +769,17 @@ int launch_sign_tiles(const SignLaunch &l, cudaStream_t stream) {
     a.stage = l.stage;
     a.slice_begin = l.slice_begin;
     a.recs = l.recs;
+    a.error = l.error;
     const uint64_t items = l.n_tiles * l.n_replicas;
     const uint64_t want = (items + SIGN_THREADS / 32 - 1) / (SIGN_THREADS / 32);
     int grid = l.grid;
     if ((uint64_t)grid > want) grid = (int)want;
-    sign_tiles_direct<<<grid, SIGN_THREADS, 0, stream>>>(a);
+    switch (l.variant) {
+        case 3: read_probe<<<grid, SIGN_THREADS, 0, stream>>>(a); break;
+        case 2: sign_tiles_ring<<<grid, SIGN_THREADS, RING_SMEM, stream>>>(a); break;
+        case 1: sign_tiles_direct<1><<<grid, SIGN_THREADS, 0, stream>>>(a); break;
+        default: sign_tiles_direct<0><<<grid, SIGN_THREADS, 0, stream>>>(a); break;
+    }
     SCOUT_CUDA(cudaGetLastError());
     return SCOUT_OK;
 }

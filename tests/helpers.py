@@ -61,22 +61,27 @@ def expected_from_patches(w, chunks):
 
 # ---- CUDA path plumbing (imported lazily so CPU-only runs never load it) -----
 
-def gpu_plan(w, chunk_bytes=None, tags=None, tile_bytes=None):
+def gpu_plan(w, chunk_bytes=None, tags=None, tile_bytes=None, variant=None):
     from paper_2608_11034_b200 import binding
     tags = shape_tags(w) if tags is None else tags
     plan = binding.Plan(w.R, binding.make_tensor_table(w.specs, tags),
                         w.chunk_bytes if chunk_bytes is None else chunk_bytes)
     if tile_bytes is not None:
         binding.scout_plan_set(plan.handle, "tile_bytes", tile_bytes)
+    if variant is not None:
+        binding.scout_plan_set(plan.handle, "variant", variant)
     return plan
 
 
-def gpu_sign_vote(w, views, chunk_bytes=None, tags=None, tile_bytes=None, caps=(4096, 4096)):
+def gpu_sign_vote(w, views, chunk_bytes=None, tags=None, tile_bytes=None, caps=(4096, 4096),
+                  variant=None):
     """-> fetch() dict of the CUDA path over device-resident views[r][t]."""
-    plan = gpu_plan(w, chunk_bytes, tags, tile_bytes)
+    from paper_2608_11034_b200 import binding
+    plan = gpu_plan(w, chunk_bytes, tags, tile_bytes, variant)
     plan.bind(views)
     plan.sign_and_vote(*caps)
     out = plan.fetch()
+    assert binding.scout_plan_get(plan.handle, "device_error") == 0
     plan.close()
     return out
 

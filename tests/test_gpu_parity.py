@@ -20,8 +20,12 @@ def _binding():
     return binding
 
 
-def _compare_everything(w, views, chunk_bytes=None, tile_bytes=None):
-    gpu = helpers.gpu_sign_vote(w, views, chunk_bytes=chunk_bytes, tile_bytes=tile_bytes)
+VARIANTS = [0, 1, 2]      # direct loads, register prefetch, bulk-async ring
+
+
+def _compare_everything(w, views, chunk_bytes=None, tile_bytes=None, variant=None):
+    gpu = helpers.gpu_sign_vote(w, views, chunk_bytes=chunk_bytes, tile_bytes=tile_bytes,
+                                variant=variant)
     host_views = [[v.cpu() for v in rep] for rep in views]
     osigs, chunks = helpers.oracle_sign_all(w, host_views, chunk_bytes=chunk_bytes)
     helpers.assert_sigs_match(gpu["sigs"], osigs, helpers.chunk_abs_sums(w, host_views, chunks))
@@ -36,10 +40,11 @@ def _compare_everything(w, views, chunk_bytes=None, tile_bytes=None):
 @pytest.mark.parametrize("cfg,case", [(1, "clean"), (1, "default"), (2, "clean"), (2, "mantissa"),
                                       (2, "split22"), (2, "split211"), (3, "default"),
                                       (4, "default"), (5, "default")])
-def test_scaled_workloads(cfg, case):
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_scaled_workloads(cfg, case, variant):
     w = inputs.workload(cfg, case, SMALL[cfg])
     _, views = inputs.generate(w, "cuda")
-    gpu, _, chunks = _compare_everything(w, views)
+    gpu, _, chunks = _compare_everything(w, views, variant=variant)
     want_out, want_und = helpers.expected_from_patches(w, chunks)
     assert gpu["outliers"] == want_out and gpu["undecided"] == want_und
 
@@ -61,8 +66,9 @@ def _odd_workload(dtype, seed):
 
 
 @pytest.mark.parametrize("dtype", ["u8", "f32", "bf16", "i64", "f16", "f64", "i32"])
-@pytest.mark.parametrize("tile_bytes", [2048, 4096])
-def test_every_dtype_and_ragged_sizes(dtype, tile_bytes):
+@pytest.mark.parametrize("tile_bytes,variant", [(2048, 0), (4096, 0), (4096, 1), (8192, 1),
+                                                (4096, 2), (8192, 2), (32768, 2)])
+def test_every_dtype_and_ragged_sizes(dtype, tile_bytes, variant):
     w = _odd_workload(dtype, 77)
     _, views = inputs.generate(w, "cuda")
     rng = random.Random(5)
@@ -70,10 +76,11 @@ def test_every_dtype_and_ragged_sizes(dtype, tile_bytes):
                               1 << rng.randrange(8 * inputs.DTYPE_BYTES[dtype]))
                  for t, s in enumerate(w.specs) if t % 2 == 0]
     inputs.apply_patches(views, w.specs, w.patches)
-    _compare_everything(w, views, tile_bytes=tile_bytes)
+    _compare_everything(w, views, tile_bytes=tile_bytes, variant=variant)
 
 
-def test_non_finite_elements():
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_non_finite_elements(variant):
     w = inputs.workload(3, "clean", SMALL[3])
     _, views = inputs.generate(w, "cuda")
     n0 = w.specs[0].numel
@@ -83,7 +90,7 @@ def test_non_finite_elements():
                  inputs.Patch(4, 1, 101, "set", 0x7F81),          # NaN with the smallest payload
                  inputs.Patch(6, 2, 7, "set", 0x7F7F)]            # largest finite bf16: no count
     inputs.apply_patches(views, w.specs, w.patches)
-    gpu, osigs, _ = _compare_everything(w, views)
+    gpu, osigs, _ = _compare_everything(w, views, variant=variant)
     assert int(gpu["sigs"]["nan_count"].sum()) == 2 and int(gpu["sigs"]["inf_count"].sum()) == 2
 
     for dtype, pats in (("f32", [0x7FC00000, 0x7F800000, 0xFF800001, 0x7F7FFFFF]),
@@ -94,8 +101,40 @@ def test_non_finite_elements():
         _, views = inputs.generate(w, "cuda")
         w.patches = [inputs.Patch(i % 3, len(w.specs) - 1 - i, i, "set", p) for i, p in enumerate(pats)]
         inputs.apply_patches(views, w.specs, w.patches)
-        gpu, _, _ = _compare_everything(w, views)
+        gpu, _, _ = _compare_everything(w, views, variant=variant)
         assert int(gpu["sigs"]["nan_count"].sum()) == 2 and int(gpu["sigs"]["inf_count"].sum()) == 1
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_bf16_subnormals_zeros_and_tiny_values(variant):
+    """The bf16 fast path widens part of the elements by bit placement, which is
+    exact for zeros and normal values; tiles whose squares are all tiny must fall
+    back to the exact loop, all-zero tiles must not."""
+    n = 40_000
+    specs = [inputs.TensorSpec(name, (n,), "bf16", "normal", 1.0)
+             for name in ("subnormal", "zeros", "tiny", "mixed", "negzero")]
+    w = inputs.Workload("bf16_small_magnitudes", 0, "x", 3, 16384, specs, 123)
+    flats, views = inputs.generate(w, "cuda")
+    g = torch.Generator(device="cuda").manual_seed(7)
+    for r in range(w.R):
+        iv = [v.view(torch.int16) for v in views[r]]
+        if r == 0:
+            pat = torch.randint(0, 0x80, (n,), generator=g, device="cuda", dtype=torch.int32)
+            sign = torch.randint(0, 2, (n,), generator=g, device="cuda", dtype=torch.int32) << 15
+            sub = ((pat | sign) & 0xFFFF).to(torch.int32)
+            sub = torch.where(sub >= 0x8000, sub - 0x10000, sub).to(torch.int16)
+            tiny = torch.randint(0x0080, 0x0400, (n,), generator=g, device="cuda", dtype=torch.int32).to(torch.int16)
+            mixed = views[r][3].view(torch.int16).clone()
+            mixed[::3] = sub[::3]
+            mixed[1::7] = 0
+            first = (sub, torch.zeros(n, dtype=torch.int16, device="cuda"), tiny, mixed,
+                     torch.full((n,), -0x8000, dtype=torch.int16, device="cuda"))
+        for dst, src in zip(iv, first):
+            dst.copy_(src)
+    gpu, osigs, chunks = _compare_everything(w, views, variant=variant)
+    assert (osigs["sumsq"][osigs["sumsq"] > 0] < 1e-60).any()      # the tiny-square case is present
+    for t in (1, 4):                                               # +0 and -0 tensors: exactly zero
+        assert (gpu["sigs"]["sumsq"][chunks["tensor"] == t] == 0).all()
 
 
 def test_huge_finite_values_take_the_classifying_path_and_stay_exact():
@@ -169,8 +208,8 @@ def test_results_are_bitwise_reproducible_and_independent_of_tiling():
     a = helpers.gpu_sign_vote(w, views)
     b = helpers.gpu_sign_vote(w, views)
     assert a["sigs"].tobytes() == b["sigs"].tobytes()
-    for tile in (2048, 8192, 32768, 65536):
-        c = helpers.gpu_sign_vote(w, views, tile_bytes=tile)
+    for tile, variant in ((2048, 0), (8192, 1), (32768, 2), (65536, 2), (65536, 1)):
+        c = helpers.gpu_sign_vote(w, views, tile_bytes=tile, variant=variant)
         assert (c["sigs"]["hash"] == a["sigs"]["hash"]).all()
         assert c["outliers"] == a["outliers"]
         assert np.allclose(c["sigs"]["sumsq"], a["sigs"]["sumsq"], rtol=1e-13, atol=0)
