@@ -246,24 +246,18 @@ def main():
     import numpy as np
     import torch
     import torch.distributed as dist
-    from paper_2608_11034_b200 import binding, inputs
+    from paper_2608_11034_b200 import binding, dist_util, inputs
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = dist_util.rank_info()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (the product path has no CPU fallback)")
     torch.cuda.set_device(local)
     if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
+        dist_util.init("nccl", torch.device("cuda", local))
+    barrier = dist_util.barrier
 
     w = inputs.workload(args.config, "default", args.scale)
-    w.seed += 4096 * rank                    # every rank scans its own replica set
+    w.seed = dist_util.rank_seed(w.seed, rank)   # every rank scans its own replica set
     flats, views = inputs.generate(w, "cuda")
     total_bytes = w.R * w.bytes_per_replica
     small = total_bytes < (1 << 30)          # working set may sit in L2: flush between steps
@@ -309,11 +303,7 @@ def main():
     clocks = sampler.stop() if sampler else None
     if not scan_ns:
         scan_ns.append(binding.scout_plan_get(plan.handle, "last_sign_ns"))
-    ms = sum(a.elapsed_time(b) for a, b in ev)
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = dist_util.max_over_ranks(sum(a.elapsed_time(b) for a, b in ev), "cuda")
 
     # the last timed step must have produced the right answer
     want = expected_pairs(w, plan.handle, binding, inputs)
@@ -328,7 +318,7 @@ def main():
     if not verified:
         raise SystemExit(f"wrong result: outliers {got[:8]} expected {want[:8]}")
 
-    value = world * total_bytes * args.steps / (ms * 1e-3) / 1e9
+    value = dist_util.aggregate_gbs(total_bytes, world, args.steps, ms)
     peak, peak_kind = measured_peak()
     scan_s = (sum(scan_ns) / len(scan_ns)) * 1e-9
     achieved = total_bytes / scan_s / 1e9

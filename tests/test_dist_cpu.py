@@ -1,0 +1,61 @@
+"""World-size-2 gloo run of the multi-rank plumbing bench.py uses: independent
+replica sets per rank, barrier, max-over-ranks timing, whole-job aggregation.
+The data path itself has no collective (each rank votes over its own replicas),
+so every rank also runs the oracle pipeline on its own shard."""
+import os
+import socket
+
+import torch.multiprocessing as mp
+
+import helpers  # noqa: F401  (puts the repository root on sys.path for the children)
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    import torch.distributed as dist
+    from oracle import scout_oracle as orc
+    from paper_2608_11034_b200 import dist_util, inputs
+    import helpers as h
+
+    assert dist_util.rank_info() == (rank, world, rank)
+    dist_util.init("gloo")
+    w = inputs.workload(1, "default", 1 / 16)
+    w.seed = dist_util.rank_seed(w.seed, rank)
+    _, views = inputs.generate(w)
+    sigs, chunks = h.oracle_sign_all(w, views, nthreads=1)
+    got = orc.vote(sigs)
+    assert got["outliers"] == h.expected_from_patches(w, chunks)[0]
+    dist_util.barrier()
+    ms_local = 10.0 + 5.0 * rank                     # rank 1 is the slow one
+    ms = dist_util.max_over_ranks(ms_local)
+    value = dist_util.aggregate_gbs(w.R * w.bytes_per_replica, world, 4, ms)
+    out.put((rank, ms, value, int(sigs["hash"][0, 0])))
+    dist_util.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_gloo():
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(out.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    (r0, ms0, v0, h0), (r1, ms1, v1, h1) = res
+    assert (r0, r1) == (0, 1)
+    assert ms0 == ms1 == 15.0                         # the max over ranks, on every rank
+    assert v0 == v1
+    bytes_per_rank = 3 * 4 * 65536
+    assert abs(v0 - 2 * bytes_per_rank * 4 / 15e-3 / 1e9) < 1e-12
+    assert h0 != h1                                   # different replica sets per rank
