@@ -155,10 +155,16 @@ def scout_consensus_vote(R: int, n_chunks: int, d_sigs: int, d_status: int, d_bi
            "scout_consensus_vote")
 
 
+_certify_buffers = {}
+
+
 def _certify_common(fn, name, plan, second, outlier_cap, undecided_cap):
-    rep = np.zeros(1, dtype=REPORT_DTYPE)
-    outl = np.zeros(max(outlier_cap, 1), dtype=OUTLIER_DTYPE)
-    und = np.zeros(max(undecided_cap, 1), dtype=np.uint64)
+    key = (outlier_cap, undecided_cap)
+    if key not in _certify_buffers:      # host landing buffers, reused between calls
+        _certify_buffers[key] = (np.zeros(1, dtype=REPORT_DTYPE),
+                                 np.zeros(max(outlier_cap, 1), dtype=OUTLIER_DTYPE),
+                                 np.zeros(max(undecided_cap, 1), dtype=np.uint64))
+    rep, outl, und = _certify_buffers[key]
     rc = _check(fn(plan, second, rep.ctypes.data, outl.ctypes.data, outlier_cap, und.ctypes.data,
                    undecided_cap), name, allow=(ERR_TRUNCATED,))
     r = {k: int(rep[0][k]) for k in REPORT_DTYPE.names}
@@ -238,7 +244,11 @@ class Plan:
             scout_plan_destroy(self.handle)
             self.handle = None
 
-    __del__ = close
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:       # interpreter shutdown: module globals may be gone
+            pass
 
     def bind(self, views) -> None:
         """views[r][t]: torch CUDA tensors (kept alive by the plan)."""

@@ -34,6 +34,15 @@ static uint32_t dtype_size(uint32_t d) {
 
 using namespace scout;
 
+// Pinned landing area of scout_certify's device-to-host copies.
+constexpr uint64_t CERTIFY_HEAD = 64;
+struct CertifyHost {
+    CertifyOut out;
+    uint32_t dev_err, pad;
+    scout_outlier_t outliers[CERTIFY_HEAD];
+    uint64_t undecided[CERTIFY_HEAD];
+};
+
 struct scout_plan {
     uint32_t R = 0;
     uint64_t T = 0, chunk_bytes = 0;
@@ -59,7 +68,8 @@ struct scout_plan {
     uint64_t *d_bitmap = nullptr, *d_majority = nullptr, *d_undecided = nullptr;
     scout_outlier_t *d_outliers = nullptr;
     uint64_t outlier_cap = 0, undecided_cap = 0;
-    CertifyOut *d_out = nullptr, *h_out = nullptr;
+    CertifyOut *d_out = nullptr;
+    CertifyHost *h_out = nullptr;  // pinned
     bool have_results = false;
 
     // host-replica staging
@@ -149,7 +159,7 @@ int ensure_certify_buffers(scout_plan *p, uint64_t outlier_cap, uint64_t undecid
         SCOUT_CUDA(cudaMalloc(&p->d_bitmap, C * sizeof(uint64_t)));
         SCOUT_CUDA(cudaMalloc(&p->d_majority, C * sizeof(uint64_t)));
         SCOUT_CUDA(cudaMalloc(&p->d_out, sizeof(CertifyOut)));
-        SCOUT_CUDA(cudaMallocHost(&p->h_out, sizeof(CertifyOut)));
+        SCOUT_CUDA(cudaMallocHost(&p->h_out, sizeof(CertifyHost)));
     }
     if (!p->d_outliers || outlier_cap > p->outlier_cap) {
         if (p->d_outliers) cudaFree(p->d_outliers);
@@ -177,18 +187,33 @@ int vote_and_report(scout_plan *p, cudaStream_t stream, scout_report_t *report,
     if (rc) return rc;
     rc = launch_certificate(C, p->d_majority, p->d_out, stream);
     if (rc) return rc;
-    SCOUT_CUDA(cudaMemcpyAsync(p->h_out, p->d_out, sizeof(CertifyOut), cudaMemcpyDeviceToHost, stream));
+    // One round trip in the common case: the counters, the error flag and the head of
+    // both lists are copied speculatively; longer lists need a second copy.
+    CertifyHost *hh = p->h_out;
+    const uint64_t head_out = std::min<uint64_t>(outlier_cap, CERTIFY_HEAD);
+    const uint64_t head_und = std::min<uint64_t>(undecided_cap, CERTIFY_HEAD);
+    SCOUT_CUDA(cudaMemcpyAsync(&hh->out, p->d_out, sizeof(CertifyOut), cudaMemcpyDeviceToHost, stream));
+    SCOUT_CUDA(cudaMemcpyAsync(&hh->dev_err, p->d_error, sizeof(uint32_t), cudaMemcpyDeviceToHost, stream));
+    if (head_out)
+        SCOUT_CUDA(cudaMemcpyAsync(hh->outliers, p->d_outliers, head_out * sizeof(scout_outlier_t),
+                                   cudaMemcpyDeviceToHost, stream));
+    if (head_und)
+        SCOUT_CUDA(cudaMemcpyAsync(hh->undecided, p->d_undecided, head_und * sizeof(uint64_t),
+                                   cudaMemcpyDeviceToHost, stream));
     SCOUT_CUDA(cudaStreamSynchronize(stream));
-    const CertifyOut &o = *p->h_out;
+    const CertifyOut &o = hh->out;
     const uint64_t n_out = std::min<uint64_t>(o.counts[4], outlier_cap);
     const uint64_t n_und = std::min<uint64_t>(o.counts[5], undecided_cap);
-    if (n_out)
-        SCOUT_CUDA(cudaMemcpyAsync(h_outliers, p->d_outliers, n_out * sizeof(scout_outlier_t),
-                                   cudaMemcpyDeviceToHost, stream));
-    if (n_und)
-        SCOUT_CUDA(cudaMemcpyAsync(h_undecided, p->d_undecided, n_und * sizeof(uint64_t),
-                                   cudaMemcpyDeviceToHost, stream));
-    if (n_out || n_und) SCOUT_CUDA(cudaStreamSynchronize(stream));
+    std::memcpy(h_outliers, hh->outliers, std::min(n_out, head_out) * sizeof(scout_outlier_t));
+    std::memcpy(h_undecided, hh->undecided, std::min(n_und, head_und) * sizeof(uint64_t));
+    if (n_out > head_out)
+        SCOUT_CUDA(cudaMemcpyAsync(h_outliers + head_out, p->d_outliers + head_out,
+                                   (n_out - head_out) * sizeof(scout_outlier_t), cudaMemcpyDeviceToHost,
+                                   stream));
+    if (n_und > head_und)
+        SCOUT_CUDA(cudaMemcpyAsync(h_undecided + head_und, p->d_undecided + head_und,
+                                   (n_und - head_und) * sizeof(uint64_t), cudaMemcpyDeviceToHost, stream));
+    if (n_out > head_out || n_und > head_und) SCOUT_CUDA(cudaStreamSynchronize(stream));
     // device lists are in arrival order; the host lists are canonical
     std::sort(h_outliers, h_outliers + n_out, [](const scout_outlier_t &a, const scout_outlier_t &b) {
         return a.chunk != b.chunk ? a.chunk < b.chunk : a.replica < b.replica;
@@ -206,10 +231,7 @@ int vote_and_report(scout_plan *p, cudaStream_t stream, scout_report_t *report,
     report->verdict = o.counts[3] ? SCOUT_UNDECIDED
                                   : (o.counts[2] ? SCOUT_VERDICT_ATTRIBUTED : SCOUT_CERTIFIED);
     p->have_results = true;
-    uint32_t dev_err = 0;
-    SCOUT_CUDA(cudaMemcpyAsync(&dev_err, p->d_error, sizeof(dev_err), cudaMemcpyDeviceToHost, stream));
-    SCOUT_CUDA(cudaStreamSynchronize(stream));
-    if (dev_err) {
+    if (hh->dev_err) {
         set_cuda_error(cudaErrorUnknown, "scan kernel: a bounded wait for a bulk copy gave up");
         return SCOUT_ERR_CUDA;
     }
@@ -474,7 +496,7 @@ int scout_plan_results(const scout_plan_t *p, const scout_sig_t **d_sigs, const 
 
 int scout_plan_replica_bad_counts(const scout_plan_t *p, uint64_t *h_counts) {
     if (!p || !h_counts || !p->have_results) return SCOUT_ERR_INVALID;
-    for (uint32_t r = 0; r < p->R; ++r) h_counts[r] = p->h_out->replica_bad[r];
+    for (uint32_t r = 0; r < p->R; ++r) h_counts[r] = p->h_out->out.replica_bad[r];
     return SCOUT_OK;
 }
 

@@ -48,6 +48,8 @@ struct Acc {
     double s0, s1, q0, q1;
 };
 
+// Streaming 16-byte load: read-only path, no L1 allocation (the data is used once).
+// .cs, L2::256B prefetch and evict-first hints measured the same on B200.
 __device__ __forceinline__ uint4 ld_stream16(const void *p) {
     uint4 v;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -234,42 +236,16 @@ __device__ __noinline__ void rescan_classifying(const uint8_t *tile, uint32_t nb
     inf_count = a.inf_count;
 }
 
-// h <- h * P + (m0 w0 + m1 w1 + m2 w2 + m3 w3) mod 2^64.
-#ifndef SCOUT_FOLD_IMPL
-#define SCOUT_FOLD_IMPL 1
-#endif
+// h <- h * P + (m0 w0 + m1 w1 + m2 w2 + m3 w3) mod 2^64.  Starting the chain from
+// h * P lets every product be a 32x32+64 multiply-add (measured: fewest
+// instructions of the forms tried; a 64-bit accumulate costs two issue slots).
 __device__ __forceinline__ void fold_row(uint64_t &h, const uint4 &v, const uint32_t (&m)[4]) {
-#if SCOUT_FOLD_IMPL == 0
-    uint64_t s = (uint64_t)m[0] * v.x;
-    s += (uint64_t)m[1] * v.y;
-    s += (uint64_t)m[2] * v.z;
-    s += (uint64_t)m[3] * v.w;
-    h = h * HASH_P + s;
-#elif SCOUT_FOLD_IMPL == 1
     uint64_t t = h * HASH_P;
     t += (uint64_t)m[0] * v.x;
     t += (uint64_t)m[1] * v.y;
     t += (uint64_t)m[2] * v.z;
     t += (uint64_t)m[3] * v.w;
     h = t;
-#elif SCOUT_FOLD_IMPL == 2
-    uint64_t t = h * HASH_P;
-    asm("mad.wide.u32 %0, %1, %2, %0;" : "+l"(t) : "r"(m[0]), "r"(v.x));
-    asm("mad.wide.u32 %0, %1, %2, %0;" : "+l"(t) : "r"(m[1]), "r"(v.y));
-    asm("mad.wide.u32 %0, %1, %2, %0;" : "+l"(t) : "r"(m[2]), "r"(v.z));
-    asm("mad.wide.u32 %0, %1, %2, %0;" : "+l"(t) : "r"(m[3]), "r"(v.w));
-    h = t;
-#else
-    // explicit 32-bit pieces: low/high words of h*P by hand, products by mad.wide
-    const uint32_t hl = (uint32_t)h, hh = (uint32_t)(h >> 32);
-    const uint32_t pl = (uint32_t)HASH_P, ph = (uint32_t)(HASH_P >> 32);
-    uint64_t t = (uint64_t)hl * pl;
-    uint32_t thi = (uint32_t)(t >> 32) + hl * ph + hh * pl;
-    t = ((uint64_t)thi << 32) | (uint32_t)t;
-    uint64_t sa = (uint64_t)m[0] * v.x + (uint64_t)m[1] * v.y;
-    uint64_t sb = (uint64_t)m[2] * v.z + (uint64_t)m[3] * v.w;
-    h = t + sa + sb;
-#endif
 }
 
 // Per-lane state of one tile's scan: the lane's four slot multipliers, its share
@@ -462,8 +438,18 @@ __global__ void __launch_bounds__(SIGN_THREADS, PREFETCH ? SCOUT_MINBLOCKS_PF : 
 // the bytes in flight do not depend on how long the arithmetic takes.  There is
 // no block-wide synchronisation: warps are independent.  Only whole rows go
 // through the ring; a chunk's ragged last row is read with plain loads.
-constexpr int RING_PIECE = 4096;  // 8 rows
-constexpr int RING_STAGES = 3;
+#ifndef SCOUT_RING_PIECE
+#define SCOUT_RING_PIECE 4096
+#endif
+#ifndef SCOUT_RING_STAGES
+#define SCOUT_RING_STAGES 3
+#endif
+#ifndef SCOUT_RING_BLOCKS
+#define SCOUT_RING_BLOCKS 2
+#endif
+constexpr int RING_PIECE = SCOUT_RING_PIECE;  // bytes per piece: whole rows
+constexpr int RING_STAGES = SCOUT_RING_STAGES;
+constexpr int RING_ROWS = RING_PIECE / (int)ROW_BYTES;
 constexpr int RING_WARPS = SIGN_THREADS / 32;
 constexpr int RING_SMEM = RING_WARPS * RING_STAGES * RING_PIECE + RING_WARPS * RING_STAGES * 8;
 constexpr uint32_t RING_WAIT_LIMIT = 1u << 24;  // polls before a wait gives up
@@ -502,134 +488,160 @@ __device__ __forceinline__ uint4 lds16(uint32_t addr) {
     return v;
 }
 
-// The next piece the copy engine should fetch for this warp.
-struct PieceCursor {
-    uint64_t item;          // index into the warp's item sequence (global item id)
-    const uint8_t *base;    // tile address
-    uint32_t full_bytes;    // whole rows of the tile, in bytes
-    uint32_t offset;        // next byte of the tile to request
-    bool valid;
+// What the ring needs to know about one work item.
+struct RingTile {
+    const uint8_t *base;
+    TileRec *rec;
+    uint32_t nbytes, dtype;
+};
+
+struct RingCtx {
+    const SignArgs &a;
+    uint64_t n_items, n_warps;
+    uint32_t lane, data0, bar0;
+    uint32_t issued, consumed;
+    // producer side: the tile whose pieces are being requested, and the one after it
+    RingTile p_cur, p_next;
+    uint64_t p_item;       // item id of p_next
+    uint32_t p_off, p_full;
+    bool p_valid;
+    bool gave_up;
+
+    __device__ __forceinline__ RingTile describe(uint64_t item) const {
+        RingTile t;
+        t.base = nullptr; t.rec = nullptr; t.nbytes = 0; t.dtype = 0;
+        if (item < n_items) {
+            const uint32_t rr = (uint32_t)(item / a.n_tiles);
+            const uint64_t ti = a.tile_begin + (item - (uint64_t)rr * a.n_tiles);
+            const uint32_t r = a.replica_begin + rr;
+            const TileDesc td = a.tiles[ti];
+            t.base = tile_address(a, td, r);
+            t.rec = &a.recs[(uint64_t)r * a.tiles_per_replica + ti];
+            t.nbytes = td.nbytes;
+            t.dtype = td.dtype;
+        }
+        return t;
+    }
+    // make p_cur the next tile that has whole rows; p_next is read one tile early so
+    // that its descriptor has arrived by the time the producer needs it
+    __device__ __forceinline__ void producer_advance() {
+        for (;;) {
+            p_cur = p_next;
+            p_valid = p_item < n_items;
+            if (!p_valid) return;
+            p_item += n_warps;
+            p_next = describe(p_item);
+            p_off = 0;
+            p_full = (p_cur.nbytes / ROW_BYTES) * ROW_BYTES;
+            if (p_full) return;
+        }
+    }
+    __device__ __forceinline__ void request() {
+        const uint32_t stage = issued % RING_STAGES;
+        const uint32_t bytes = min((uint32_t)RING_PIECE, p_full - p_off);
+        if (lane == 0) {
+            mbar_expect_tx(bar0 + 8 * stage, bytes);
+            bulk_g2s(data0 + stage * RING_PIECE, p_cur.base + p_off, bytes, bar0 + 8 * stage);
+        }
+        ++issued;
+        p_off += bytes;
+        if (p_off >= p_full) producer_advance();
+    }
+    // wait for the oldest outstanding piece; false if the bounded wait gave up
+    __device__ __forceinline__ bool acquire(uint32_t &saddr) {
+        const uint32_t stage = consumed % RING_STAGES;
+        const uint32_t parity = (consumed / RING_STAGES) & 1u;
+        uint32_t polls = 0;
+        while (!mbar_try_wait(bar0 + 8 * stage, parity)) {
+            if (++polls > RING_WAIT_LIMIT) { gave_up = true; return false; }
+        }
+        saddr = data0 + stage * RING_PIECE + 16u * lane;
+        return true;
+    }
+    __device__ __forceinline__ void release() {
+        __syncwarp();  // every lane has read the piece before it is requested again
+        ++consumed;
+        if (p_valid) request();
+    }
 };
 
 template <int DT>
-__device__ __forceinline__ void fold_piece(TileScan<DT> &st, uint32_t saddr, uint32_t rows) {
-    if (rows == RING_PIECE / ROW_BYTES) {
+__device__ __forceinline__ void ring_tile(RingCtx &c, const RingTile &t, TileRec &rec) {
+    TileScan<DT> st;
+    st.begin(c.lane);
+    uint32_t rows = t.nbytes / ROW_BYTES;
+#pragma unroll 1
+    for (; rows >= RING_ROWS; rows -= RING_ROWS) {
+        uint32_t saddr;
+        if (!c.acquire(saddr)) return;
+        uint4 v[RING_ROWS];
 #pragma unroll
-        for (int r = 0; r < RING_PIECE / (int)ROW_BYTES; ++r) st.row(lds16(saddr + r * ROW_BYTES));
-    } else {
-        for (uint32_t r = 0; r < rows; ++r) st.row(lds16(saddr + r * ROW_BYTES));
+        for (int r = 0; r < RING_ROWS; ++r) v[r] = lds16(saddr + r * ROW_BYTES);
+#pragma unroll
+        for (int r = 0; r < RING_ROWS; ++r) st.row(v[r]);
+        c.release();
     }
+    if (rows) {
+        uint32_t saddr;
+        if (!c.acquire(saddr)) return;
+        for (uint32_t r = 0; r < rows; ++r) st.row(lds16(saddr + r * ROW_BYTES));
+        c.release();
+    }
+    st.finish(t.base, t.nbytes, c.lane, rec);
 }
 
-__global__ void __launch_bounds__(SIGN_THREADS, 2) sign_tiles_ring(const SignArgs a) {
+__global__ void __launch_bounds__(SIGN_THREADS, SCOUT_RING_BLOCKS) sign_tiles_ring(const SignArgs a) {
     extern __shared__ __align__(128) uint8_t ring_smem[];
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t wib = threadIdx.x >> 5;
     const uint64_t warp = (uint64_t)blockIdx.x * RING_WARPS + wib;
-    const uint64_t n_warps = (uint64_t)gridDim.x * RING_WARPS;
-    const uint64_t n_items = a.n_tiles * a.n_replicas;
-    const uint32_t data0 = smem_u32(ring_smem) + wib * (RING_STAGES * RING_PIECE);
-    const uint32_t bar0 = smem_u32(ring_smem) + RING_WARPS * RING_STAGES * RING_PIECE + wib * (RING_STAGES * 8);
+    RingCtx c{a};
+    c.n_items = a.n_tiles * a.n_replicas;
+    c.n_warps = (uint64_t)gridDim.x * RING_WARPS;
+    c.lane = lane;
+    c.data0 = smem_u32(ring_smem) + wib * (RING_STAGES * RING_PIECE);
+    c.bar0 = smem_u32(ring_smem) + RING_WARPS * RING_STAGES * RING_PIECE + wib * (RING_STAGES * 8);
+    c.issued = c.consumed = 0;
+    c.gave_up = false;
 
     if (lane == 0) {
 #pragma unroll
-        for (int s = 0; s < RING_STAGES; ++s) mbar_init(bar0 + 8 * s, 1);
+        for (int s = 0; s < RING_STAGES; ++s) mbar_init(c.bar0 + 8 * s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncwarp();
 
-    auto locate = [&](uint64_t item, TileDesc &td, uint32_t &r, uint64_t &t) {
-        const uint32_t rr = (uint32_t)(item / a.n_tiles);
-        t = a.tile_begin + (item - (uint64_t)rr * a.n_tiles);
-        r = a.replica_begin + rr;
-        td = a.tiles[t];
-    };
-    // move the cursor to the first item at or after `item` that has whole rows
-    auto seek = [&](PieceCursor &c, uint64_t item) {
-        c.valid = false;
-        for (; item < n_items; item += n_warps) {
-            TileDesc td;
-            uint32_t r;
-            uint64_t t;
-            locate(item, td, r, t);
-            const uint32_t fb = (td.nbytes / ROW_BYTES) * ROW_BYTES;
-            if (fb) {
-                c.item = item;
-                c.base = tile_address(a, td, r);
-                c.full_bytes = fb;
-                c.offset = 0;
-                c.valid = true;
-                return;
-            }
-        }
-    };
-    uint32_t issued = 0;  // pieces requested so far; piece n lives in stage n % RING_STAGES
-    auto request = [&](PieceCursor &c) {
-        const uint32_t stage = issued % RING_STAGES;
-        const uint32_t bytes = min((uint32_t)RING_PIECE, c.full_bytes - c.offset);
-        if (lane == 0) {
-            mbar_expect_tx(bar0 + 8 * stage, bytes);
-            bulk_g2s(data0 + stage * RING_PIECE, c.base + c.offset, bytes, bar0 + 8 * stage);
-        }
-        ++issued;
-        c.offset += bytes;
-        if (c.offset >= c.full_bytes) seek(c, c.item + n_warps);
-    };
+    c.p_item = warp;
+    c.p_next = c.describe(warp);
+    c.producer_advance();
+    for (int s = 0; s < RING_STAGES && c.p_valid; ++s) c.request();
 
-    PieceCursor cur;
-    seek(cur, warp);
-    for (int s = 0; s < RING_STAGES && cur.valid; ++s) request(cur);
-
-    uint32_t consumed = 0;
-    bool gave_up = false;
-    for (uint64_t item = warp; item < n_items && !gave_up; item += n_warps) {
-        TileDesc td;
-        uint32_t r;
-        uint64_t t;
-        locate(item, td, r, t);
-        const uint8_t *tile = tile_address(a, td, r);
-        const uint32_t full_rows = td.nbytes / ROW_BYTES;
+    RingTile next = c.describe(warp);
+#pragma unroll 1
+    for (uint64_t item = warp; item < c.n_items && !c.gave_up; item += c.n_warps) {
+        const RingTile t = next;
+        next = c.describe(item + c.n_warps);  // in flight while this tile is folded
         TileRec rec;
-        auto run = [&](auto tag) {
-            constexpr int DT = decltype(tag)::value;
-            TileScan<DT> st;
-            st.begin(lane);
-            for (uint32_t row0 = 0; row0 < full_rows; row0 += RING_PIECE / ROW_BYTES) {
-                const uint32_t stage = consumed % RING_STAGES;
-                const uint32_t parity = (consumed / RING_STAGES) & 1u;
-                uint32_t polls = 0;
-                while (!mbar_try_wait(bar0 + 8 * stage, parity)) {
-                    if (++polls > RING_WAIT_LIMIT) { gave_up = true; break; }
-                }
-                if (gave_up) break;
-                const uint32_t rows = min((uint32_t)(RING_PIECE / ROW_BYTES), full_rows - row0);
-                fold_piece<DT>(st, data0 + stage * RING_PIECE + 16u * lane, rows);
-                __syncwarp();  // every lane has read the piece before it is requested again
-                ++consumed;
-                if (cur.valid) request(cur);
-            }
-            if (!gave_up) st.finish(tile, td.nbytes, lane, rec);
-        };
-        switch (td.dtype) {
-            case SCOUT_DT_F32:  run(std::integral_constant<int, SCOUT_DT_F32>{}); break;
-            case SCOUT_DT_BF16: run(std::integral_constant<int, SCOUT_DT_BF16>{}); break;
-            case SCOUT_DT_I64:  run(std::integral_constant<int, SCOUT_DT_I64>{}); break;
-            case SCOUT_DT_F16:  run(std::integral_constant<int, SCOUT_DT_F16>{}); break;
-            case SCOUT_DT_F64:  run(std::integral_constant<int, SCOUT_DT_F64>{}); break;
-            case SCOUT_DT_I32:  run(std::integral_constant<int, SCOUT_DT_I32>{}); break;
-            default:            run(std::integral_constant<int, SCOUT_DT_U8>{}); break;
+        switch (t.dtype) {
+            case SCOUT_DT_F32:  ring_tile<SCOUT_DT_F32>(c, t, rec); break;
+            case SCOUT_DT_BF16: ring_tile<SCOUT_DT_BF16>(c, t, rec); break;
+            case SCOUT_DT_I64:  ring_tile<SCOUT_DT_I64>(c, t, rec); break;
+            case SCOUT_DT_F16:  ring_tile<SCOUT_DT_F16>(c, t, rec); break;
+            case SCOUT_DT_F64:  ring_tile<SCOUT_DT_F64>(c, t, rec); break;
+            case SCOUT_DT_I32:  ring_tile<SCOUT_DT_I32>(c, t, rec); break;
+            default:            ring_tile<SCOUT_DT_U8>(c, t, rec); break;
         }
-        if (!gave_up && lane == 0) store_record(&a.recs[(uint64_t)r * a.tiles_per_replica + t], rec);
+        if (!c.gave_up && lane == 0) store_record(t.rec, rec);
     }
-    if (gave_up) {
+    if (c.gave_up) {
         // A copy never completed.  Report it, give the copies still in flight one more
         // bounded chance to land (shared memory must not be released under them), return.
         if (lane == 0 && a.error) atomicExch(a.error, 1u);
-        for (uint32_t n = consumed; n < issued; ++n) {
+        for (uint32_t n = c.consumed; n < c.issued; ++n) {
             const uint32_t stage = n % RING_STAGES, parity = (n / RING_STAGES) & 1u;
             uint32_t polls = 0;
-            while (!mbar_try_wait(bar0 + 8 * stage, parity) && ++polls <= RING_WAIT_LIMIT) {}
+            while (!mbar_try_wait(c.bar0 + 8 * stage, parity) && ++polls <= RING_WAIT_LIMIT) {}
         }
     }
 }
