@@ -76,6 +76,16 @@ def lib():
             "scout_shape_tag": (u64, [u32, vp]),
             "scout_plan_set": (C.c_int, [vp, C.c_char_p, i64]),
             "scout_plan_get": (C.c_int, [vp, C.c_char_p, C.POINTER(i64)]),
+            "scout_ledger_create": (C.c_int, [u32, C.POINTER(vp)]),
+            "scout_ledger_destroy": (C.c_int, [vp]),
+            "scout_ledger_state": (C.c_int, [vp, vp]),
+            "scout_ledger_save": (C.c_int, [vp, C.c_int, u64, C.c_int, C.c_int, vp]),
+            "scout_ledger_retrieve": (C.c_int, [vp, C.c_int, C.c_int, C.c_int, vp]),
+            "scout_outcome_from_report": (C.c_int, [vp, C.POINTER(C.c_int)]),
+            "scout_mesh_size": (C.c_int, [vp, C.POINTER(u64)]),
+            "scout_mesh_coords": (C.c_int, [vp, u64, vp]),
+            "scout_mesh_rank": (C.c_int, [vp, vp, C.POINTER(u64)]),
+            "scout_peer_group": (C.c_int, [vp, u64, vp, u64, C.POINTER(u64), C.POINTER(C.c_int)]),
             "scout_strerror": (C.c_char_p, [C.c_int]),
             "scout_version": (C.c_int, []),
             "scout_last_cuda_error": (C.c_char_p, []),
@@ -210,6 +220,98 @@ def scout_sign_chunks_noalloc(R: int, replica_ptrs: Sequence[int], nbytes: int, 
     a = np.asarray(list(replica_ptrs), dtype=np.uint64)
     _check(lib().scout_sign_chunks_noalloc(R, a.ctypes.data, nbytes, dtype, meta_tag, chunk_bytes,
                                            d_sigs, stream), "scout_sign_chunks_noalloc")
+
+
+# ---- host-only entry points: checkpoint ledger, peer groups -----------------------
+
+OUTCOME_HEALTHY, OUTCOME_STRAGGLER, OUTCOME_SDC, OUTCOME_HANG, OUTCOME_OTHER = range(5)
+ROLE_NONE, ROLE_LATEST, ROLE_CANDIDATE, ROLE_VERIFIED = range(4)
+LEDGER_CAPTURED, LEDGER_BOUNDARY, LEDGER_RETRIEVAL, LEDGER_NEED_SWEEP = range(4)
+NO_CHECKPOINT = 2**64 - 1
+GROUP_NONE, GROUP_REPLICA, GROUP_SHARD = range(3)
+LEDGER_STATE_DTYPE = np.dtype([("latest", "<u8"), ("candidate", "<u8"), ("verified", "<u8"),
+                               ("q", "<u4"), ("K", "<u4"), ("n_persisted", "<u8")])
+LEDGER_EVENT_DTYPE = np.dtype([("action", "<i4"), ("role", "<i4"), ("checkpoint", "<u8"),
+                               ("promoted", "<u8")])
+MESH_DTYPE = np.dtype([(k, "<u4") for k in "dstpce"])
+
+
+def scout_ledger_create(K: int) -> int:
+    out = C.c_void_p()
+    _check(lib().scout_ledger_create(K, C.byref(out)), "scout_ledger_create")
+    return out.value
+
+
+def scout_ledger_destroy(ledger: int) -> None:
+    _check(lib().scout_ledger_destroy(ledger), "scout_ledger_destroy")
+
+
+def scout_ledger_state(ledger: int) -> dict:
+    st = np.zeros(1, dtype=LEDGER_STATE_DTYPE)
+    _check(lib().scout_ledger_state(ledger, st.ctypes.data), "scout_ledger_state")
+    return {k: int(st[0][k]) for k in LEDGER_STATE_DTYPE.names}
+
+
+def _event(ev) -> dict:
+    return {k: int(ev[0][k]) for k in LEDGER_EVENT_DTYPE.names}
+
+
+def scout_ledger_save(ledger: int, outcome: int, captured: int, machines_accessible: bool = True,
+                      sweep_has_sdc: int = -1) -> dict:
+    ev = np.zeros(1, dtype=LEDGER_EVENT_DTYPE)
+    _check(lib().scout_ledger_save(ledger, outcome, captured, int(machines_accessible),
+                                   sweep_has_sdc, ev.ctypes.data), "scout_ledger_save")
+    return _event(ev)
+
+
+def scout_ledger_retrieve(ledger: int, failure: int, machines_accessible: bool = True,
+                          sweep_has_sdc: int = -1) -> dict:
+    ev = np.zeros(1, dtype=LEDGER_EVENT_DTYPE)
+    _check(lib().scout_ledger_retrieve(ledger, failure, int(machines_accessible), sweep_has_sdc,
+                                       ev.ctypes.data), "scout_ledger_retrieve")
+    return _event(ev)
+
+
+def scout_outcome_from_report(report: dict) -> int:
+    rep = np.zeros(1, dtype=REPORT_DTYPE)
+    for k in REPORT_DTYPE.names:
+        rep[0][k] = report[k]
+    out = C.c_int()
+    _check(lib().scout_outcome_from_report(rep.ctypes.data, C.byref(out)), "scout_outcome_from_report")
+    return out.value
+
+
+def _mesh(shape) -> np.ndarray:
+    m = np.zeros(1, dtype=MESH_DTYPE)
+    m[0] = tuple(shape)
+    return m
+
+
+def scout_mesh_size(shape) -> int:
+    n, m = C.c_uint64(), _mesh(shape)
+    _check(lib().scout_mesh_size(m.ctypes.data, C.byref(n)), "scout_mesh_size")
+    return n.value
+
+
+def scout_mesh_coords(shape, rank: int):
+    out, m = np.zeros(1, dtype=MESH_DTYPE), _mesh(shape)
+    _check(lib().scout_mesh_coords(m.ctypes.data, rank, out.ctypes.data), "scout_mesh_coords")
+    return tuple(int(out[0][k]) for k in "dstpce")
+
+
+def scout_mesh_rank(shape, coords) -> int:
+    r, m, at = C.c_uint64(), _mesh(shape), _mesh(coords)
+    _check(lib().scout_mesh_rank(m.ctypes.data, at.ctypes.data, C.byref(r)), "scout_mesh_rank")
+    return r.value
+
+
+def scout_peer_group(shape, rank: int, cap: int = 4096):
+    """-> (kind, peers) with peers in bitmap order"""
+    peers = np.zeros(max(cap, 1), dtype=np.uint64)
+    n, kind, m = C.c_uint64(), C.c_int(), _mesh(shape)
+    _check(lib().scout_peer_group(m.ctypes.data, rank, peers.ctypes.data, cap, C.byref(n),
+                                  C.byref(kind)), "scout_peer_group", allow=(ERR_TRUNCATED,))
+    return kind.value, [int(x) for x in peers[:min(n.value, cap)]]
 
 
 def scout_version() -> int:

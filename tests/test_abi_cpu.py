@@ -19,7 +19,8 @@ def lib():
 
 
 def test_every_declared_symbol_is_exported(lib):
-    header = open(os.path.join(ROOT, "include", "scout.h")).read()
+    inc = os.path.join(ROOT, "include")
+    header = "".join(open(os.path.join(inc, h)).read() for h in sorted(os.listdir(inc)))
     names = set(re.findall(r"SCOUT_API[^;(]*?\b(scout_\w+)\s*\(", header))
     assert {"scout_sign_chunks", "scout_consensus_vote", "scout_certify", "scout_plan_create",
             "scout_plan_bind", "scout_plan_destroy"} <= names
