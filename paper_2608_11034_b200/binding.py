@@ -86,6 +86,7 @@ def lib():
             "scout_mesh_coords": (C.c_int, [vp, u64, vp]),
             "scout_mesh_rank": (C.c_int, [vp, vp, C.POINTER(u64)]),
             "scout_peer_group": (C.c_int, [vp, u64, vp, u64, C.POINTER(u64), C.POINTER(C.c_int)]),
+            "scout_consensus_timing": (C.c_int, [u32, u64, vp, C.c_double, vp, vp, vp, vp, vp]),
             "scout_strerror": (C.c_char_p, [C.c_int]),
             "scout_version": (C.c_int, []),
             "scout_last_cuda_error": (C.c_char_p, []),
@@ -220,6 +221,12 @@ def scout_sign_chunks_noalloc(R: int, replica_ptrs: Sequence[int], nbytes: int, 
     a = np.asarray(list(replica_ptrs), dtype=np.uint64)
     _check(lib().scout_sign_chunks_noalloc(R, a.ctypes.data, nbytes, dtype, meta_tag, chunk_bytes,
                                            d_sigs, stream), "scout_sign_chunks_noalloc")
+
+
+def scout_consensus_timing(N: int, G: int, d_times: int, kappa: float, d_status: int,
+                           d_bitmap: int, d_median: int, d_scale: int, stream: int) -> None:
+    _check(lib().scout_consensus_timing(N, G, d_times, kappa, d_status, d_bitmap, d_median,
+                                        d_scale, stream), "scout_consensus_timing")
 
 
 # ---- host-only entry points: checkpoint ledger, peer groups -----------------------
