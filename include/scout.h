@@ -59,6 +59,8 @@ enum { SCOUT_AGREE = 0, SCOUT_ATTRIBUTED = 1, SCOUT_INCONCLUSIVE = 2 };
 /* Verdict of scout_certify over a whole replicated state. */
 enum { SCOUT_CERTIFIED = 0, SCOUT_VERDICT_ATTRIBUTED = 1, SCOUT_UNDECIDED = 2 };
 
+#define SCOUT_MAX_REPLICAS 1024 /* signing and scout_consensus_vote_wide; one-word bitmaps stop at 64 */
+
 typedef struct scout_plan scout_plan_t; /* opaque; owns its device tables and scratch */
 
 /* Comparable evidence of one (chunk, replica) (Sec. 5.2).  Only `hash` is
@@ -99,9 +101,14 @@ typedef struct {
  * chunk is this library's unit of evidence: C3 is applied once per chunk, so a
  * disagreement is localised to (replica, chunk) instead of (replica, tensor)
  * as in Sec. 5.2.
- *   R            number of replicas, 2..64 (a singleton has no comparison,
- *                Sec. 4 "Peer-group size"; more than 64 needs a wider bitmap:
- *                SCOUT_ERR_UNSUPPORTED)
+ *   R            number of replicas bound to this plan, 1..SCOUT_MAX_REPLICAS.
+ *                2..64: everything.  65..1024: scout_sign_chunks and
+ *                scout_consensus_vote_wide (multi-word bitmaps; the paper's peer
+ *                groups reach degree 192); scout_certify returns
+ *                SCOUT_ERR_UNSUPPORTED.  1: signing only - the local step when
+ *                every GPU holds one replica and the records are gathered
+ *                afterwards; a singleton has no comparison (Sec. 4 "Peer-group
+ *                size"), so voting or certifying with R < 2 is SCOUT_ERR_INVALID.
  *   T, tensors   host array of T descriptors, copied
  *   chunk_bytes  a multiple of 512, at most 1 GiB
  *   out          receives the plan; destroy with scout_plan_destroy
@@ -147,6 +154,21 @@ SCOUT_API int scout_consensus_vote(uint32_t R, uint64_t C, const scout_sig_t *d_
                          uint64_t *d_bitmap, scout_outlier_t *d_outliers, uint64_t outlier_cap,
                          uint64_t *d_undecided, uint64_t undecided_cap, uint64_t *d_counts,
                          void *stream);
+
+/* The same rule for groups of up to SCOUT_MAX_REPLICAS peers and for records that
+ * were gathered from one GPU per replica.  The record of (chunk c, replica r) is
+ * d_sigs[c * chunk_stride + r * replica_stride] (strides in records):
+ * (R, 1) is the chunk-major table scout_sign_chunks writes; (1, C) is the
+ * rank-major table an AllGather of per-rank [C] records produces (Algorithm 1
+ * line 2), so no transposition is needed.  d_bitmap: device [C][W] words with
+ * W = ceil(R / 64), bit (r mod 64) of word (r / 64) for replica r; may be NULL.
+ * Everything else as in scout_consensus_vote. */
+SCOUT_API int scout_consensus_vote_wide(uint32_t R, uint64_t C, const scout_sig_t *d_sigs,
+                                        uint64_t chunk_stride, uint64_t replica_stride,
+                                        uint8_t *d_status, uint64_t *d_bitmap,
+                                        scout_outlier_t *d_outliers, uint64_t outlier_cap,
+                                        uint64_t *d_undecided, uint64_t undecided_cap,
+                                        uint64_t *d_counts, void *stream);
 
 /* ---- certify a replicated state -------------------------------------------
  * sign + vote + roll-up over everything bound to the plan (the optimizer-

@@ -331,6 +331,55 @@ int orc_vote(uint32_t R, uint64_t C, const orc_sig_t *sigs, uint8_t *status, uin
     return (n_out > outlier_cap || n_und > undecided_cap) ? -6 : 0;
 }
 
+/* The same rule for groups of any size and for strided record tables: the
+ * record of (chunk c, replica r) is sigs[c * chunk_stride + r * replica_stride];
+ * bitmap holds W = ceil(R / 64) words per chunk. */
+int orc_vote_wide(uint32_t R, uint64_t C, const orc_sig_t *sigs, uint64_t chunk_stride,
+                  uint64_t replica_stride, uint8_t *status, uint64_t *bitmap, orc_outlier_t *outliers,
+                  uint64_t outlier_cap, uint64_t *undecided, uint64_t undecided_cap, uint64_t *counts)
+{
+    if (R < 2) return -1;
+    uint32_t W = (R + 63) / 64;
+    uint64_t n_agree = 0, n_attr = 0, n_inc = 0, n_out = 0, n_und = 0;
+    for (uint64_t c = 0; c < C; ++c) {
+        const orc_sig_t *row = sigs + c * chunk_stride;
+        uint32_t best_count = 0;
+        uint64_t best_value = 0;
+        for (uint32_t j = 0; j < R; ++j) {
+            uint32_t cnt = 0;
+            for (uint32_t i = 0; i < R; ++i)
+                if (row[i * replica_stride].hash == row[j * replica_stride].hash) ++cnt;
+            if (cnt > best_count) { best_count = cnt; best_value = row[j * replica_stride].hash; }
+        }
+        for (uint32_t w = 0; w < W; ++w) bitmap[c * W + w] = 0;
+        if (2ull * best_count <= (uint64_t)R) {
+            status[c] = ORC_INCONCLUSIVE;
+            ++n_inc;
+            if (n_und < undecided_cap) undecided[n_und] = c;
+            ++n_und;
+            continue;
+        }
+        uint32_t marked = 0;
+        for (uint32_t j = 0; j < R; ++j) {
+            if (row[j * replica_stride].hash != best_value) {
+                bitmap[c * W + j / 64] |= 1ull << (j % 64);
+                if (n_out < outlier_cap) {
+                    outliers[n_out].chunk = c;
+                    outliers[n_out].replica = j;
+                    outliers[n_out].reserved = 0;
+                }
+                ++n_out;
+                ++marked;
+            }
+        }
+        status[c] = marked ? ORC_ATTRIBUTED : ORC_AGREE;
+        if (marked) ++n_attr; else ++n_agree;
+    }
+    counts[0] = C; counts[1] = n_agree; counts[2] = n_attr; counts[3] = n_inc;
+    counts[4] = n_out; counts[5] = n_und;
+    return (n_out > outlier_cap || n_und > undecided_cap) ? -6 : 0;
+}
+
 /* ---- roll-ups ------------------------------------------------------------ */
 
 /* Tensor-level signature from the chunk hashes of one replica, in order. */

@@ -110,6 +110,12 @@ int orc_vote(uint32_t R, uint64_t C, const orc_sig_t *sigs, uint8_t *status, uin
              orc_outlier_t *outliers, uint64_t outlier_cap, uint64_t *undecided,
              uint64_t undecided_cap, uint64_t *counts);
 
+/* orc_vote for any group size and strided tables: record (c, r) at
+ * sigs[c*chunk_stride + r*replica_stride]; bitmap has ceil(R/64) words per chunk */
+int orc_vote_wide(uint32_t R, uint64_t C, const orc_sig_t *sigs, uint64_t chunk_stride,
+                  uint64_t replica_stride, uint8_t *status, uint64_t *bitmap, orc_outlier_t *outliers,
+                  uint64_t outlier_cap, uint64_t *undecided, uint64_t undecided_cap, uint64_t *counts);
+
 uint64_t orc_rollup(const uint64_t *hashes, uint64_t n);
 /* certificate over the majority hash of every chunk, in order */
 uint64_t orc_certificate(uint32_t R, uint64_t C, const orc_sig_t *sigs, const uint8_t *status,

@@ -80,6 +80,9 @@ def lib():
         L.orc_vote.restype = C.c_int
         L.orc_vote.argtypes = [C.c_uint32, C.c_uint64, vp, vp, vp, vp, C.c_uint64, vp,
                                C.c_uint64, vp]
+        L.orc_vote_wide.restype = C.c_int
+        L.orc_vote_wide.argtypes = [C.c_uint32, C.c_uint64, vp, C.c_uint64, C.c_uint64, vp, vp, vp,
+                                    C.c_uint64, vp, C.c_uint64, vp]
         L.orc_rollup.restype = C.c_uint64
         L.orc_rollup.argtypes = [vp, C.c_uint64]
         L.orc_certificate.restype = C.c_uint64
@@ -189,6 +192,27 @@ def vote(sigs: np.ndarray, outlier_cap: int | None = None, undecided_cap: int | 
     return dict(status=status, bitmap=bitmap,
                 outliers=[(int(o["chunk"]), int(o["replica"])) for o in outl[:no]],
                 undecided=[int(x) for x in und[:nu]], counts=[int(x) for x in counts], rc=rc)
+
+
+def vote_wide(sigs: np.ndarray, R: int, Cn: int, chunk_stride: int, replica_stride: int):
+    """Vote over a flat record table with strides (in records); any R >= 2.
+    -> dict(status, bitmap [C, W], outliers, undecided, counts, rc)"""
+    assert sigs.dtype == SIG_DTYPE
+    flat = np.ascontiguousarray(sigs).reshape(-1)
+    W = (R + 63) // 64
+    status = np.zeros(Cn, dtype=np.uint8)
+    bitmap = np.zeros((Cn, W), dtype=np.uint64)
+    outl = np.zeros(max(Cn * R, 1), dtype=OUTLIER_DTYPE)
+    und = np.zeros(max(Cn, 1), dtype=np.uint64)
+    counts = np.zeros(6, dtype=np.uint64)
+    rc = lib().orc_vote_wide(R, Cn, flat.ctypes.data, chunk_stride, replica_stride, status.ctypes.data,
+                             bitmap.ctypes.data, outl.ctypes.data, Cn * R, und.ctypes.data, Cn,
+                             counts.ctypes.data)
+    if rc == -1:
+        raise ValueError("orc_vote_wide: invalid arguments")
+    return dict(status=status, bitmap=bitmap,
+                outliers=[(int(o["chunk"]), int(o["replica"])) for o in outl[:int(counts[4])]],
+                undecided=[int(x) for x in und[:int(counts[5])]], counts=[int(x) for x in counts], rc=rc)
 
 
 def rollup(hashes) -> int:

@@ -67,6 +67,7 @@ def lib():
             "scout_plan_destroy": (C.c_int, [vp]),
             "scout_sign_chunks": (C.c_int, [vp, vp, vp]),
             "scout_consensus_vote": (C.c_int, [u32, u64, vp, vp, vp, vp, u64, vp, u64, vp, vp]),
+            "scout_consensus_vote_wide": (C.c_int, [u32, u64, vp, u64, u64, vp, vp, vp, u64, vp, u64, vp, vp]),
             "scout_certify": (C.c_int, [vp, vp, vp, vp, u64, vp, u64]),
             "scout_plan_results": (C.c_int, [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)]),
             "scout_plan_replica_bad_counts": (C.c_int, [vp, vp]),
@@ -167,6 +168,16 @@ def scout_consensus_vote(R: int, n_chunks: int, d_sigs: int, d_status: int, d_bi
 
 
 _certify_buffers = {}
+
+
+def scout_consensus_vote_wide(R: int, n_chunks: int, d_sigs: int, chunk_stride: int,
+                              replica_stride: int, d_status: int, d_bitmap: int, d_outliers: int,
+                              outlier_cap: int, d_undecided: int, undecided_cap: int, d_counts: int,
+                              stream: int) -> None:
+    _check(lib().scout_consensus_vote_wide(R, n_chunks, d_sigs, chunk_stride, replica_stride, d_status,
+                                           d_bitmap, d_outliers, outlier_cap, d_undecided,
+                                           undecided_cap, d_counts, stream),
+           "scout_consensus_vote_wide")
 
 
 def _certify_common(fn, name, plan, second, outlier_cap, undecided_cap):

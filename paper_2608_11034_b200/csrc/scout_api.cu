@@ -246,8 +246,8 @@ int scout_plan_create(uint32_t R, uint64_t T, const scout_tensor_t *tensors, uin
                       scout_plan_t **out) {
     if (!out) return SCOUT_ERR_INVALID;
     *out = nullptr;
-    if (R < 2 || !tensors || T == 0) return SCOUT_ERR_INVALID;
-    if (R > 64) return SCOUT_ERR_UNSUPPORTED;
+    if (R < 1 || !tensors || T == 0) return SCOUT_ERR_INVALID;
+    if (R > SCOUT_MAX_REPLICAS) return SCOUT_ERR_UNSUPPORTED;
     if (chunk_bytes == 0 || chunk_bytes % ROW_BYTES != 0 || chunk_bytes > (1ull << 30))
         return SCOUT_ERR_INVALID;
     if (T > 0xFFFFFFFFull) return SCOUT_ERR_UNSUPPORTED;
@@ -403,9 +403,22 @@ int scout_consensus_vote(uint32_t R, uint64_t C, const scout_sig_t *d_sigs, uint
                        undecided_cap, d_counts, nullptr, nullptr, (cudaStream_t)stream);
 }
 
+int scout_consensus_vote_wide(uint32_t R, uint64_t C, const scout_sig_t *d_sigs, uint64_t chunk_stride,
+                              uint64_t replica_stride, uint8_t *d_status, uint64_t *d_bitmap,
+                              scout_outlier_t *d_outliers, uint64_t outlier_cap, uint64_t *d_undecided,
+                              uint64_t undecided_cap, uint64_t *d_counts, void *stream) {
+    if (R < 2) return SCOUT_ERR_INVALID;
+    if (R > SCOUT_MAX_REPLICAS) return SCOUT_ERR_UNSUPPORTED;
+    if (!d_counts || (C && !d_sigs) || chunk_stride == 0 || replica_stride == 0) return SCOUT_ERR_INVALID;
+    if ((outlier_cap && !d_outliers) || (undecided_cap && !d_undecided)) return SCOUT_ERR_INVALID;
+    return launch_vote_wide(R, C, d_sigs, chunk_stride, replica_stride, d_status, d_bitmap, d_outliers,
+                            outlier_cap, d_undecided, undecided_cap, d_counts, (cudaStream_t)stream);
+}
+
 int scout_certify(scout_plan_t *p, void *stream, scout_report_t *report, scout_outlier_t *h_outliers,
                   uint64_t outlier_cap, uint64_t *h_undecided, uint64_t undecided_cap) {
-    if (!p || !report || !p->bound) return SCOUT_ERR_INVALID;
+    if (!p || !report || !p->bound || p->R < 2) return SCOUT_ERR_INVALID;
+    if (p->R > 64) return SCOUT_ERR_UNSUPPORTED;
     if ((outlier_cap && !h_outliers) || (undecided_cap && !h_undecided)) return SCOUT_ERR_INVALID;
     int rc = ensure_certify_buffers(p, outlier_cap, undecided_cap);
     if (rc) return rc;
@@ -417,7 +430,8 @@ int scout_certify(scout_plan_t *p, void *stream, scout_report_t *report, scout_o
 int scout_certify_host(scout_plan_t *p, const void *const *h_ptrs, scout_report_t *report,
                        scout_outlier_t *h_outliers, uint64_t outlier_cap, uint64_t *h_undecided,
                        uint64_t undecided_cap) {
-    if (!p || !h_ptrs || !report) return SCOUT_ERR_INVALID;
+    if (!p || !h_ptrs || !report || p->R < 2) return SCOUT_ERR_INVALID;
+    if (p->R > 64) return SCOUT_ERR_UNSUPPORTED;
     if ((outlier_cap && !h_outliers) || (undecided_cap && !h_undecided)) return SCOUT_ERR_INVALID;
     const uint64_t n = (uint64_t)p->R * p->T;
     for (uint64_t i = 0; i < n; ++i)

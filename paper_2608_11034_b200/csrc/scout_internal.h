@@ -137,6 +137,10 @@ int launch_vote(uint32_t R, uint64_t C, const scout_sig_t *d_sigs, uint8_t *d_st
                 uint64_t *d_bitmap, scout_outlier_t *d_outliers, uint64_t outlier_cap,
                 uint64_t *d_undecided, uint64_t undecided_cap, uint64_t *d_counts,
                 uint64_t *d_majority, CertifyOut *d_out, cudaStream_t stream);
+int launch_vote_wide(uint32_t R, uint64_t C, const scout_sig_t *d_sigs, uint64_t chunk_stride,
+                     uint64_t replica_stride, uint8_t *d_status, uint64_t *d_bitmap,
+                     scout_outlier_t *d_outliers, uint64_t outlier_cap, uint64_t *d_undecided,
+                     uint64_t undecided_cap, uint64_t *d_counts, cudaStream_t stream);
 int launch_certificate(uint64_t C, const uint64_t *d_majority, CertifyOut *d_out,
                        cudaStream_t stream);
 int launch_rollup_tensors(const ChunkDesc *chunks, const uint64_t *tensor_chunk0, uint64_t T,

@@ -114,6 +114,96 @@ __global__ void __launch_bounds__(VOTE_THREADS) vote_chunks(
     }
 }
 
+// Wide groups (up to SCOUT_MAX_REPLICAS peers) and strided record tables: one CTA
+// per chunk.  The R hashes go to shared memory; thread j counts the peers that
+// hold e_j; a block-wide maximum gives c*; 2 c* <= R is Inconclusive; otherwise
+// the value of any thread whose count is c* is e* and the bitmap words are
+// assembled from warp ballots.
+constexpr int WIDE_THREADS = 128;
+
+__global__ void __launch_bounds__(WIDE_THREADS) vote_chunks_wide(
+    uint32_t R, uint64_t C, const scout_sig_t *__restrict__ sigs, uint64_t chunk_stride,
+    uint64_t replica_stride, uint8_t *status_out, uint64_t *bitmap_out, scout_outlier_t *outliers,
+    uint64_t outlier_cap, uint64_t *undecided, uint64_t undecided_cap, uint64_t *counts) {
+    __shared__ uint64_t e[SCOUT_MAX_REPLICAS];
+    __shared__ uint32_t bits[SCOUT_MAX_REPLICAS / 32];
+    __shared__ uint32_t best_count, n_set;
+    __shared__ unsigned long long best_value, list_base;
+    const uint32_t tid = threadIdx.x, lane = tid & 31u;
+    const uint32_t W = (R + 63u) / 64u;
+    uint32_t n_agree = 0, n_attr = 0, n_inc = 0;  // kept by thread 0
+
+    for (uint64_t c = blockIdx.x; c < C; c += gridDim.x) {
+        for (uint32_t r = tid; r < R; r += WIDE_THREADS)
+            e[r] = sigs[c * chunk_stride + (uint64_t)r * replica_stride].hash;
+        if (tid == 0) { best_count = 0; n_set = 0; }
+        for (uint32_t w = tid; w < SCOUT_MAX_REPLICAS / 32; w += WIDE_THREADS) bits[w] = 0u;
+        __syncthreads();
+        uint32_t mine = 0;
+        uint64_t mine_value = 0;
+        for (uint32_t r = tid; r < R; r += WIDE_THREADS) {
+            const uint64_t v = e[r];
+            uint32_t cnt = 0;
+            for (uint32_t i = 0; i < R; ++i) cnt += (e[i] == v);
+            if (cnt > mine) { mine = cnt; mine_value = v; }
+        }
+        atomicMax(&best_count, mine);
+        __syncthreads();
+        const uint32_t best = best_count;
+        const bool decided = 2u * best > R;
+        if (decided && mine == best) best_value = mine_value;  // every writer holds the same e*
+        __syncthreads();
+        if (decided) {
+            const uint64_t majority = best_value;
+            for (uint32_t r0 = 0; r0 < R; r0 += WIDE_THREADS) {  // uniform trip count: ballots are safe
+                const uint32_t r = r0 + tid;
+                const uint32_t b = __ballot_sync(0xFFFFFFFFu, r < R && e[r] != majority);
+                if (lane == 0 && b) {
+                    bits[r >> 5] = b;
+                    atomicAdd(&n_set, (uint32_t)__popc(b));
+                }
+            }
+        }
+        __syncthreads();
+        const uint32_t total = n_set;
+        if (tid == 0) {
+            const uint32_t st = !decided ? SCOUT_INCONCLUSIVE : (total ? SCOUT_ATTRIBUTED : SCOUT_AGREE);
+            if (status_out) status_out[c] = (uint8_t)st;
+            if (st == SCOUT_INCONCLUSIVE) {
+                ++n_inc;
+                const unsigned long long pos = atomicAdd((unsigned long long *)&counts[5], 1ull);
+                if (pos < undecided_cap) undecided[pos] = c;
+            } else if (total) {
+                ++n_attr;
+                list_base = atomicAdd((unsigned long long *)&counts[4], (unsigned long long)total);
+            } else {
+                ++n_agree;
+            }
+        }
+        if (bitmap_out)
+            for (uint32_t w = tid; w < W; w += WIDE_THREADS)
+                bitmap_out[c * W + w] = ((uint64_t)bits[2 * w + 1] << 32) | bits[2 * w];
+        __syncthreads();
+        if (total) {  // block-aggregated append: one atomic per chunk, offsets from the bit words
+            for (uint32_t r = tid; r < R; r += WIDE_THREADS) {
+                if ((bits[r >> 5] >> (r & 31u)) & 1u) {
+                    uint32_t before = __popc(bits[r >> 5] & ((1u << (r & 31u)) - 1u));
+                    for (uint32_t w = 0; w < (r >> 5); ++w) before += __popc(bits[w]);
+                    const uint64_t pos = list_base + before;
+                    if (pos < outlier_cap) outliers[pos] = scout_outlier_t{c, r, 0u};
+                }
+            }
+        }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        if (n_agree) atomicAdd((unsigned long long *)&counts[1], (unsigned long long)n_agree);
+        if (n_attr) atomicAdd((unsigned long long *)&counts[2], (unsigned long long)n_attr);
+        if (n_inc) atomicAdd((unsigned long long *)&counts[3], (unsigned long long)n_inc);
+        if (blockIdx.x == 0) counts[0] = C;
+    }
+}
+
 // Certificate: a <- mix64(seed ^ C); a <- mix64(a ^ majority_c) for every chunk
 // in order.  The chain is sequential by construction; one warp streams the
 // hashes in coalesced groups of 32 and lane 0 runs the chain.
@@ -165,6 +255,20 @@ int launch_vote(uint32_t R, uint64_t C, const scout_sig_t *d_sigs, uint8_t *d_st
     vote_chunks<<<(int)blocks, VOTE_THREADS, 0, stream>>>(R, C, d_sigs, d_status, d_bitmap, d_outliers,
                                                          outlier_cap, d_undecided, undecided_cap,
                                                          d_counts, d_majority, d_out);
+    SCOUT_CUDA(cudaGetLastError());
+    return SCOUT_OK;
+}
+
+int launch_vote_wide(uint32_t R, uint64_t C, const scout_sig_t *d_sigs, uint64_t chunk_stride,
+                     uint64_t replica_stride, uint8_t *d_status, uint64_t *d_bitmap,
+                     scout_outlier_t *d_outliers, uint64_t outlier_cap, uint64_t *d_undecided,
+                     uint64_t undecided_cap, uint64_t *d_counts, cudaStream_t stream) {
+    SCOUT_CUDA(cudaMemsetAsync(d_counts, 0, 6 * sizeof(uint64_t), stream));
+    uint64_t blocks = C < 148ull * 8 ? C : 148ull * 8;
+    if (blocks == 0) blocks = 1;
+    vote_chunks_wide<<<(int)blocks, WIDE_THREADS, 0, stream>>>(R, C, d_sigs, chunk_stride, replica_stride,
+                                                               d_status, d_bitmap, d_outliers, outlier_cap,
+                                                               d_undecided, undecided_cap, d_counts);
     SCOUT_CUDA(cudaGetLastError());
     return SCOUT_OK;
 }

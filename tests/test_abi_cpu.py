@@ -47,8 +47,8 @@ def test_plan_arguments_are_validated_before_any_device_work():
     t = np.zeros(1, dtype=binding.TENSOR_DTYPE)
     t[0] = (1024, binding.DT_F32, 0, 0)
     bad = [
-        (1, t, 512, binding.ERR_INVALID),        # a singleton group has no comparison
-        (65, t, 512, binding.ERR_UNSUPPORTED),   # bitmap is one 64-bit word
+        (0, t, 512, binding.ERR_INVALID),
+        (1025, t, 512, binding.ERR_UNSUPPORTED),  # beyond the widest supported peer group
         (3, t, 0, binding.ERR_INVALID),
         (3, t, 1000, binding.ERR_INVALID),       # chunk size must be a multiple of 512
         (3, t, (1 << 30) + 512, binding.ERR_INVALID),
@@ -70,3 +70,7 @@ def test_vote_arguments_are_validated(lib):
     assert lib.scout_consensus_vote(65, 1, 8, 0, 0, 0, 0, 0, 0, 8, 0) == binding.ERR_UNSUPPORTED
     assert lib.scout_consensus_vote(3, 1, 8, 0, 0, 0, 0, 0, 0, 0, 0) == binding.ERR_INVALID
     assert lib.scout_consensus_vote(3, 1, 8, 0, 0, 0, 5, 0, 0, 8, 0) == binding.ERR_INVALID
+    # a singleton has no comparison, whatever the bitmap width
+    assert lib.scout_consensus_vote_wide(1, 1, 8, 1, 1, 0, 0, 0, 0, 0, 0, 8, 0) == binding.ERR_INVALID
+    assert lib.scout_consensus_vote_wide(1025, 1, 8, 1025, 1, 0, 0, 0, 0, 0, 0, 8, 0) == binding.ERR_UNSUPPORTED
+    assert lib.scout_consensus_vote_wide(3, 1, 8, 0, 1, 0, 0, 0, 0, 0, 0, 8, 0) == binding.ERR_INVALID

@@ -59,3 +59,50 @@ def test_two_ranks_gloo():
     bytes_per_rank = 3 * 4 * 65536
     assert abs(v0 - 2 * bytes_per_rank * 4 / 15e-3 / 1e9) < 1e-12
     assert h0 != h1                                   # different replica sets per rank
+
+
+def _gather_worker(rank, world, port, out):
+    """One replica per rank: sign locally (oracle), all-gather the records, vote
+    locally; every rank must reach the same result without a coordinator."""
+    os.environ.update(RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from oracle import scout_oracle as orc
+    from paper_2608_11034_b200 import dist_util, inputs
+    import helpers as h
+
+    dist_util.init("gloo")
+    w = inputs.workload(1, "default", 1 / 16)
+    w.R = world
+    w.patches = [inputs.Patch(1, 0, 777, "xor", 1 << 4)]
+    _, views = inputs.generate(w)                       # same seed everywhere: equivalent replicas
+    tt = h.oracle_tensor_table(w)
+    chunks = orc.chunk_table(tt, w.chunk_bytes)
+    mine = np.zeros((len(chunks), 1), dtype=orc.SIG_DTYPE)
+    orc.sign_replica(tt, [inputs.to_numpy_bytes(v) for v in views[rank]], w.chunk_bytes, mine, 0, 1)
+    local = torch.from_numpy(mine.view(np.uint8).reshape(-1).copy())
+    gathered = [torch.empty_like(local) for _ in range(world)]
+    dist.all_gather(gathered, local)                    # Algorithm 1 line 2
+    table = torch.stack(gathered).numpy().view(orc.SIG_DTYPE).reshape(world, len(chunks))
+    res = orc.vote_wide(table, world, len(chunks), 1, len(chunks))     # rank-major strides
+    out.put((rank, res["outliers"], res["undecided"], res["counts"]))
+    dist_util.barrier()
+    dist.destroy_process_group()
+
+
+def test_three_ranks_gather_and_vote_identically():
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_gather_worker, args=(r, 3, port, out)) for r in range(3)]
+    for p in procs:
+        p.start()
+    res = sorted(out.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert [r[1:] for r in res] == [res[0][1:]] * 3
+    chunk = (777 * 4) // 65536
+    assert res[0][1] == [(chunk, 1)] and res[0][2] == []

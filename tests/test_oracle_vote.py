@@ -114,3 +114,33 @@ def test_certify_rollup():
     split = _sigs([[a, a, a], [1, 2, 3]])
     rep = orc.certify(split)["report"]
     assert rep["verdict"] == 2 and rep["certificate"] == 0 and rep["n_undecided"] == 1
+
+
+def test_wide_vote_equals_the_narrow_one_and_the_counting_rule():
+    import random
+    rng = random.Random(17)
+    # R <= 64: the wide form must reproduce orc_vote, in both table layouts
+    for R in (2, 3, 5, 17, 64):
+        rows = [[rng.randrange(3) for _ in range(R)] for _ in range(60)]
+        sig = _sigs(rows)
+        narrow = orc.vote(sig)
+        for table, cs, rs in ((sig, R, 1), (np.ascontiguousarray(sig.T), 1, len(rows))):
+            wide = orc.vote_wide(table, R, len(rows), cs, rs)
+            assert (wide["status"] == narrow["status"]).all()
+            assert (wide["bitmap"][:, 0] == narrow["bitmap"]).all()
+            assert wide["outliers"] == narrow["outliers"] and wide["undecided"] == narrow["undecided"]
+            assert wide["counts"] == narrow["counts"]
+    # R > 64: against the counting rule, bit positions across words
+    for R in (65, 100, 192, 300):
+        rows = []
+        for _ in range(25):
+            row = [7] * R
+            for j in rng.sample(range(R), rng.choice([0, 1, 3, R // 2, R // 2 + 1, R - 1])):
+                row[j] = rng.choice([8, 9])
+            rows.append(row)
+        wide = orc.vote_wide(_sigs(rows), R, len(rows), R, 1)
+        for c, row in enumerate(rows):
+            s, B = defn.vote_one(row)
+            got = sum(int(w) << (64 * k) for k, w in enumerate(wide["bitmap"][c]))
+            assert (int(wide["status"][c]), got) == (s, B)
+        assert wide["outliers"] == sorted(wide["outliers"])
