@@ -462,14 +462,33 @@ int scout_certify_host(scout_plan_t *p, const void *const *h_ptrs, scout_report_
             const uint64_t b = p->tiles[t1 - 1].poff + p->tiles[t1 - 1].nbytes;
             const int buf = (int)(slice & 1);
             if (slice >= 2) SCOUT_CUDA(cudaStreamWaitEvent(p->s_copy, p->ev_done[buf], 0));
+            // One copy per run of tensors that sit in host memory exactly as in the packed
+            // image (same spacing, so only alignment padding of < 256 bytes lies between
+            // them): a replica kept as one flat buffer is copied slice by slice instead of
+            // tensor by tensor.
+            const uint8_t *run_src = nullptr;
+            uint64_t run_dst = 0, run_len = 0;
             for (uint32_t t = p->tiles[t0].tensor; t <= p->tiles[t1 - 1].tensor; ++t) {
                 const uint64_t lo = std::max<uint64_t>(a, p->tensor_poff[t]);
                 const uint64_t hi = std::min<uint64_t>(b, p->tensor_poff[t] + p->tensors[t].nbytes);
                 if (hi <= lo) continue;
                 const uint8_t *src = (const uint8_t *)h_ptrs[(uint64_t)r * p->T + t] + (lo - p->tensor_poff[t]);
-                SCOUT_CUDA(cudaMemcpyAsync(p->d_stage[buf] + (lo - a), src, hi - lo,
-                                           cudaMemcpyHostToDevice, p->s_copy));
+                const uint64_t dst = lo - a;
+                if (run_len && src - run_src == (ptrdiff_t)(dst - run_dst) && dst - run_dst >= run_len &&
+                    dst - run_dst - run_len < 256) {
+                    run_len = dst - run_dst + (hi - lo);
+                    continue;
+                }
+                if (run_len)
+                    SCOUT_CUDA(cudaMemcpyAsync(p->d_stage[buf] + run_dst, run_src, run_len,
+                                               cudaMemcpyHostToDevice, p->s_copy));
+                run_src = src;
+                run_dst = dst;
+                run_len = hi - lo;
             }
+            if (run_len)
+                SCOUT_CUDA(cudaMemcpyAsync(p->d_stage[buf] + run_dst, run_src, run_len,
+                                           cudaMemcpyHostToDevice, p->s_copy));
             SCOUT_CUDA(cudaEventRecord(p->ev_copied[buf], p->s_copy));
             SCOUT_CUDA(cudaStreamWaitEvent(p->s_comp, p->ev_copied[buf], 0));
             SignLaunch l;
