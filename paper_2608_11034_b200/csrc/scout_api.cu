@@ -86,10 +86,11 @@ struct scout_plan {
 namespace {
 
 uint32_t auto_tile_bytes(uint64_t total_bytes) {
-    // aim for several work items per resident warp; 2 KiB .. 32 KiB, power of two
-    const uint64_t want_items = 148ull * 32 * 8;
+    // About two work items per resident warp, 4 KiB .. 32 KiB, power of two (measured:
+    // 12.6 MB is fastest with 4 KiB tiles, 201 MB with 16 KiB, anything >= 1 GB with 32 KiB).
+    const uint64_t want_items = 148ull * 32 * 2;
     uint64_t t = total_bytes / want_items;
-    uint32_t tile = 2048;
+    uint32_t tile = 4096;
     while (tile < 32768 && (uint64_t)tile * 2 <= t) tile *= 2;
     return tile;
 }
@@ -127,7 +128,7 @@ int upload_tables(scout_plan *p) {
     return SCOUT_OK;
 }
 
-int sign_all(scout_plan *p, cudaStream_t stream, scout_sig_t *d_sigs) {
+int sign_all(scout_plan *p, cudaStream_t stream, scout_sig_t *d_sigs, CertifyOut *zero_out = nullptr) {
     SignLaunch l;
     l.tiles = p->d_tiles;
     l.tile_begin = 0;
@@ -148,7 +149,7 @@ int sign_all(scout_plan *p, cudaStream_t stream, scout_sig_t *d_sigs) {
     if (rc) return rc;
     if (p->timing) SCOUT_CUDA(cudaEventRecord(p->ev_t1, stream));
     return launch_finalize(p->d_chunks, p->chunks.size(), p->R, p->d_recs, p->tiles.size(),
-                           p->tile_bytes / ROW_BYTES, d_sigs, stream);
+                           p->tile_bytes / ROW_BYTES, d_sigs, zero_out, stream);
 }
 
 int ensure_certify_buffers(scout_plan *p, uint64_t outlier_cap, uint64_t undecided_cap) {
@@ -181,8 +182,9 @@ int vote_and_report(scout_plan *p, cudaStream_t stream, scout_report_t *report,
                     scout_outlier_t *h_outliers, uint64_t outlier_cap, uint64_t *h_undecided,
                     uint64_t undecided_cap) {
     const uint64_t C = p->chunks.size();
+    // the finalise kernel that precedes this on the stream cleared d_out
     int rc = launch_vote(p->R, C, p->d_sigs, p->d_status, p->d_bitmap, p->d_outliers, outlier_cap,
-                         p->d_undecided, undecided_cap, p->d_out->counts, p->d_majority, p->d_out,
+                         p->d_undecided, undecided_cap, p->d_out->counts, p->d_majority, p->d_out, true,
                          stream);
     if (rc) return rc;
     rc = launch_certificate(C, p->d_majority, p->d_out, stream);
@@ -400,7 +402,7 @@ int scout_consensus_vote(uint32_t R, uint64_t C, const scout_sig_t *d_sigs, uint
     if (!d_counts || (C && !d_sigs)) return SCOUT_ERR_INVALID;
     if ((outlier_cap && !d_outliers) || (undecided_cap && !d_undecided)) return SCOUT_ERR_INVALID;
     return launch_vote(R, C, d_sigs, d_status, d_bitmap, d_outliers, outlier_cap, d_undecided,
-                       undecided_cap, d_counts, nullptr, nullptr, (cudaStream_t)stream);
+                       undecided_cap, d_counts, nullptr, nullptr, false, (cudaStream_t)stream);
 }
 
 int scout_consensus_vote_wide(uint32_t R, uint64_t C, const scout_sig_t *d_sigs, uint64_t chunk_stride,
@@ -423,7 +425,7 @@ int scout_certify(scout_plan_t *p, void *stream, scout_report_t *report, scout_o
     int rc = ensure_certify_buffers(p, outlier_cap, undecided_cap);
     if (rc) return rc;
     cudaStream_t s = (cudaStream_t)stream;
-    if ((rc = sign_all(p, s, p->d_sigs))) return rc;
+    if ((rc = sign_all(p, s, p->d_sigs, p->d_out))) return rc;
     return vote_and_report(p, s, report, h_outliers, outlier_cap, h_undecided, undecided_cap);
 }
 
@@ -513,7 +515,7 @@ int scout_certify_host(scout_plan_t *p, const void *const *h_ptrs, scout_report_
         }
     }
     rc = launch_finalize(p->d_chunks, p->chunks.size(), p->R, p->d_recs, NT, p->tile_bytes / ROW_BYTES,
-                         p->d_sigs, p->s_comp);
+                         p->d_sigs, p->d_out, p->s_comp);
     if (rc) return rc;
     return vote_and_report(p, p->s_comp, report, h_outliers, outlier_cap, h_undecided, undecided_cap);
 }

@@ -109,6 +109,31 @@ void set_cuda_error(cudaError_t e, const char *what);
         }                                                 \
     } while (0)
 
+// ---- programmatic dependent launch ------------------------------------------------
+// The small kernels that follow the scan (finalise, vote, certificate) are launched
+// with programmatic stream serialisation: their CTAs may be scheduled while the
+// previous kernel drains, and wait at griddepcontrol.wait until that kernel has
+// completed and its writes are visible.  Without the launch attribute both
+// instructions are no-ops.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t stream,
+                                    Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- kernel launchers (defined in the .cu files) ------------------------------
 struct SignLaunch {
     const TileDesc *tiles;        // device
@@ -129,14 +154,16 @@ struct SignLaunch {
 int launch_sign_tiles(const SignLaunch &a, cudaStream_t stream);
 int sign_grid_size(int variant, int device, int *grid);
 
+// zero_out (may be null): a CertifyOut the finalise kernel clears for the vote that follows
 int launch_finalize(const ChunkDesc *chunks, uint64_t C, uint32_t R, const TileRec *recs,
                     uint64_t tiles_per_replica, uint32_t tile_rows, scout_sig_t *d_sigs,
-                    cudaStream_t stream);
+                    CertifyOut *zero_out, cudaStream_t stream);
 
 int launch_vote(uint32_t R, uint64_t C, const scout_sig_t *d_sigs, uint8_t *d_status,
                 uint64_t *d_bitmap, scout_outlier_t *d_outliers, uint64_t outlier_cap,
                 uint64_t *d_undecided, uint64_t undecided_cap, uint64_t *d_counts,
-                uint64_t *d_majority, CertifyOut *d_out, cudaStream_t stream);
+                uint64_t *d_majority, CertifyOut *d_out, bool counters_already_zero,
+                cudaStream_t stream);
 int launch_vote_wide(uint32_t R, uint64_t C, const scout_sig_t *d_sigs, uint64_t chunk_stride,
                      uint64_t replica_stride, uint8_t *d_status, uint64_t *d_bitmap,
                      scout_outlier_t *d_outliers, uint64_t outlier_cap, uint64_t *d_undecided,

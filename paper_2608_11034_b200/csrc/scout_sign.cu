@@ -412,6 +412,7 @@ __device__ __forceinline__ void store_record(TileRec *dst_rec, const TileRec &re
 // Persistent grid; every warp takes whole tiles, replica-major, round-robin.
 template <int PREFETCH>
 __global__ void __launch_bounds__(SIGN_THREADS, PREFETCH ? SCOUT_MINBLOCKS_PF : SCOUT_MINBLOCKS) sign_tiles_direct(const SignArgs a) {
+    pdl_launch_dependents();
     const uint32_t lane = threadIdx.x & 31u;
     const uint64_t warp = (uint64_t)blockIdx.x * (SIGN_THREADS / 32) + (threadIdx.x >> 5);
     const uint64_t n_warps = (uint64_t)gridDim.x * (SIGN_THREADS / 32);
@@ -694,7 +695,11 @@ __global__ void __launch_bounds__(FIN_THREADS) finalize_chunks(const ChunkDesc *
                                                                uint32_t R, const TileRec *recs,
                                                                uint64_t tiles_per_replica,
                                                                uint32_t tile_rows, uint64_t p_stride,
-                                                               scout_sig_t *sigs) {
+                                                               scout_sig_t *sigs, CertifyOut *zero_out) {
+    pdl_launch_dependents();
+    pdl_wait();
+    if (zero_out && blockIdx.x == 0 && threadIdx.x < sizeof(CertifyOut) / sizeof(uint64_t))
+        reinterpret_cast<uint64_t *>(zero_out)[threadIdx.x] = 0ull;
     const uint32_t lane = threadIdx.x & 31u;
     const uint64_t warp = (uint64_t)blockIdx.x * (FIN_THREADS / 32) + (threadIdx.x >> 5);
     const uint64_t n_warps = (uint64_t)gridDim.x * (FIN_THREADS / 32);
@@ -798,15 +803,15 @@ int launch_sign_tiles(const SignLaunch &l, cudaStream_t stream) {
 
 int launch_finalize(const ChunkDesc *chunks, uint64_t C, uint32_t R, const TileRec *recs,
                     uint64_t tiles_per_replica, uint32_t tile_rows, scout_sig_t *d_sigs,
-                    cudaStream_t stream) {
+                    CertifyOut *zero_out, cudaStream_t stream) {
     if (C == 0) return SCOUT_OK;
     const uint64_t items = C * R;
     uint64_t blocks = (items + FIN_THREADS / 32 - 1) / (FIN_THREADS / 32);
     if (blocks > 148ull * 16) blocks = 148ull * 16;
-    finalize_chunks<<<(int)blocks, FIN_THREADS, 0, stream>>>(chunks, C, R, recs, tiles_per_replica,
-                                                            tile_rows, pow_p(32ull * tile_rows),
-                                                            d_sigs);
-    SCOUT_CUDA(cudaGetLastError());
+    static_assert(sizeof(CertifyOut) / sizeof(uint64_t) <= FIN_THREADS, "one thread per word clears it");
+    SCOUT_CUDA(launch_dependent(finalize_chunks, dim3((unsigned)blocks), dim3(FIN_THREADS), stream, chunks, C,
+                                R, recs, tiles_per_replica, tile_rows, pow_p(32ull * tile_rows), d_sigs,
+                                zero_out));
     return SCOUT_OK;
 }
 

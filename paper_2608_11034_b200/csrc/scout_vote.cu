@@ -16,6 +16,8 @@ __global__ void __launch_bounds__(VOTE_THREADS) vote_chunks(
     uint32_t R, uint64_t C, const scout_sig_t *__restrict__ sigs, uint8_t *status_out,
     uint64_t *bitmap_out, scout_outlier_t *outliers, uint64_t outlier_cap, uint64_t *undecided,
     uint64_t undecided_cap, uint64_t *counts, uint64_t *majority_out, CertifyOut *cert) {
+    pdl_launch_dependents();
+    pdl_wait();
     const uint32_t lane = threadIdx.x & 31u;
     const uint64_t warp = (uint64_t)blockIdx.x * (VOTE_THREADS / 32) + (threadIdx.x >> 5);
     const uint64_t n_warps = (uint64_t)gridDim.x * (VOTE_THREADS / 32);
@@ -208,6 +210,7 @@ __global__ void __launch_bounds__(WIDE_THREADS) vote_chunks_wide(
 // in order.  The chain is sequential by construction; one warp streams the
 // hashes in coalesced groups of 32 and lane 0 runs the chain.
 __global__ void certificate_chain(uint64_t C, const uint64_t *__restrict__ majority, CertifyOut *out) {
+    pdl_wait();
     const uint32_t lane = threadIdx.x;
     uint64_t a = mix64(SEED_CERT ^ C);
     uint64_t next = lane < C ? majority[lane] : 0ull;
@@ -245,17 +248,26 @@ __global__ void rollup_tensors(const uint64_t *__restrict__ tensor_chunk0, uint6
 int launch_vote(uint32_t R, uint64_t C, const scout_sig_t *d_sigs, uint8_t *d_status,
                 uint64_t *d_bitmap, scout_outlier_t *d_outliers, uint64_t outlier_cap,
                 uint64_t *d_undecided, uint64_t undecided_cap, uint64_t *d_counts,
-                uint64_t *d_majority, CertifyOut *d_out, cudaStream_t stream) {
-    if (d_out) SCOUT_CUDA(cudaMemsetAsync(d_out, 0, sizeof(CertifyOut), stream));
-    if ((void *)d_counts != (void *)d_out)
-        SCOUT_CUDA(cudaMemsetAsync(d_counts, 0, 6 * sizeof(uint64_t), stream));
+                uint64_t *d_majority, CertifyOut *d_out, bool counters_already_zero,
+                cudaStream_t stream) {
+    if (!counters_already_zero) {
+        if (d_out) SCOUT_CUDA(cudaMemsetAsync(d_out, 0, sizeof(CertifyOut), stream));
+        if ((void *)d_counts != (void *)d_out)
+            SCOUT_CUDA(cudaMemsetAsync(d_counts, 0, 6 * sizeof(uint64_t), stream));
+    }
     uint64_t blocks = (C + VOTE_THREADS / 32 - 1) / (VOTE_THREADS / 32);
     if (blocks > 148ull * 8) blocks = 148ull * 8;
     if (blocks == 0) blocks = 1;
-    vote_chunks<<<(int)blocks, VOTE_THREADS, 0, stream>>>(R, C, d_sigs, d_status, d_bitmap, d_outliers,
-                                                         outlier_cap, d_undecided, undecided_cap,
-                                                         d_counts, d_majority, d_out);
-    SCOUT_CUDA(cudaGetLastError());
+    if (counters_already_zero) {  // follows the finalise kernel directly: dependent launch
+        SCOUT_CUDA(launch_dependent(vote_chunks, dim3((unsigned)blocks), dim3(VOTE_THREADS), stream, R, C,
+                                    d_sigs, d_status, d_bitmap, d_outliers, outlier_cap, d_undecided,
+                                    undecided_cap, d_counts, d_majority, d_out));
+    } else {
+        vote_chunks<<<(int)blocks, VOTE_THREADS, 0, stream>>>(R, C, d_sigs, d_status, d_bitmap, d_outliers,
+                                                             outlier_cap, d_undecided, undecided_cap,
+                                                             d_counts, d_majority, d_out);
+        SCOUT_CUDA(cudaGetLastError());
+    }
     return SCOUT_OK;
 }
 
@@ -274,8 +286,7 @@ int launch_vote_wide(uint32_t R, uint64_t C, const scout_sig_t *d_sigs, uint64_t
 }
 
 int launch_certificate(uint64_t C, const uint64_t *d_majority, CertifyOut *d_out, cudaStream_t stream) {
-    certificate_chain<<<1, 32, 0, stream>>>(C, d_majority, d_out);
-    SCOUT_CUDA(cudaGetLastError());
+    SCOUT_CUDA(launch_dependent(certificate_chain, dim3(1), dim3(32), stream, C, d_majority, d_out));
     return SCOUT_OK;
 }
 
