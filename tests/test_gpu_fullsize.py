@@ -172,3 +172,30 @@ def test_config_3_full_size():
     plan.close()
     del views
     _free()
+
+
+def test_largest_chunk_size_one_gib():
+    """chunk_bytes at its maximum (1 GiB): 32,768 tiles per chunk go through the
+    finaliser's strided combine; the second chunk of each tensor is one ragged row."""
+    from paper_2608_11034_b200 import binding
+    _free()
+    _need(6)
+    n = (1 << 30) + 516
+    w = inputs.Workload("one_gib_chunk", 0, "x", 2, 1 << 30,
+                        [inputs.TensorSpec("blob", (n,), "u8", "bytes"),
+                         inputs.TensorSpec("grad", ((1 << 28) + 129,), "f32", "normal", 0.02)], 99)
+    w.patches = [inputs.Patch(1, 0, (1 << 30) - 1, "xor", 0x80), inputs.Patch(0, 1, 1 << 28, "xor", 1)]
+    _, views = inputs.generate(w, "cuda")
+    plan = helpers.gpu_plan(w)
+    plan.bind(views)
+    plan.sign_and_vote()
+    got = plan.fetch()
+    chunks = plan.chunk_table()
+    assert plan.C == 4 and [int(c["nbytes"]) for c in chunks] == [1 << 30, 516, 1 << 30, 516]
+    # two replicas: a difference is detected but cannot be attributed (two-rank group)
+    assert got["outliers"] == [] and got["undecided"] == [0, 3]
+    assert list(got["status"]) == [binding.INCONCLUSIVE, binding.AGREE, binding.AGREE, binding.INCONCLUSIVE]
+    _check_sampled(w, views, got["sigs"], chunks, [(0, 1), (1, 0), (2, 0), (3, 0), (3, 1)])
+    plan.close()
+    del views
+    _free()
