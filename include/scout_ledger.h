@@ -96,6 +96,19 @@ SCOUT_API int scout_mesh_rank(const scout_mesh_t *shape, const scout_mesh_t *coo
 SCOUT_API int scout_peer_group(const scout_mesh_t *shape, uint64_t rank, uint64_t *peers /*host*/,
                                uint64_t cap, uint64_t *n, int *kind);
 
+/* ---- rotating slice (Sec. 9 "Optimizer boundary") -----------------------------
+ * The optimizer-boundary check compares a rotating 64K-element slice of each
+ * tensor instead of the whole tensor.  The paper does not say how the slice
+ * moves; this library's reading: consecutive windows of `slice_elems` elements,
+ * window `step` starting at (step mod n_windows) * slice_elems with
+ * n_windows = ceil(numel / slice_elems); the last window is short; after it the
+ * rotation starts again at element 0.  Signing a slice = a plan whose tensor is
+ * (base + begin * element_size, count * element_size).
+ *   begin, count   first element and length of the window for this step */
+#define SCOUT_DEFAULT_SLICE_ELEMS 65536u
+SCOUT_API int scout_rotating_slice(uint64_t numel, uint64_t slice_elems, uint64_t step,
+                                   uint64_t *begin, uint64_t *count);
+
 #ifdef __cplusplus
 }
 #endif

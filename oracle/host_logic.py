@@ -70,3 +70,11 @@ def peer_group(shape, r):
         peers = [q for q, a in ranks.items() if a[2:] == (t, p, c, e)]
         return "shard", sorted(peers)
     return "none", [r]
+
+
+def rotating_slice(numel, slice_elems, step):
+    """Window `step` of the rotation over a tensor of `numel` elements: the
+    windows are the consecutive pieces range(0, numel, slice_elems), visited
+    round-robin (the paper only says the slice rotates; this is the reading)."""
+    windows = [(b, min(slice_elems, numel - b)) for b in range(0, numel, slice_elems)]
+    return windows[step % len(windows)]

@@ -88,6 +88,7 @@ def lib():
             "scout_mesh_rank": (C.c_int, [vp, vp, C.POINTER(u64)]),
             "scout_peer_group": (C.c_int, [vp, u64, vp, u64, C.POINTER(u64), C.POINTER(C.c_int)]),
             "scout_consensus_timing": (C.c_int, [u32, u64, vp, C.c_double, vp, vp, vp, vp, vp]),
+            "scout_rotating_slice": (C.c_int, [u64, u64, u64, C.POINTER(u64), C.POINTER(u64)]),
             "scout_strerror": (C.c_char_p, [C.c_int]),
             "scout_version": (C.c_int, []),
             "scout_last_cuda_error": (C.c_char_p, []),
@@ -330,6 +331,14 @@ def scout_peer_group(shape, rank: int, cap: int = 4096):
     _check(lib().scout_peer_group(m.ctypes.data, rank, peers.ctypes.data, cap, C.byref(n),
                                   C.byref(kind)), "scout_peer_group", allow=(ERR_TRUNCATED,))
     return kind.value, [int(x) for x in peers[:min(n.value, cap)]]
+
+
+def scout_rotating_slice(numel: int, slice_elems: int, step: int):
+    """-> (begin, count) of the window checked at this step"""
+    b, n = C.c_uint64(), C.c_uint64()
+    _check(lib().scout_rotating_slice(numel, slice_elems, step, C.byref(b), C.byref(n)),
+           "scout_rotating_slice")
+    return b.value, n.value
 
 
 def scout_version() -> int:

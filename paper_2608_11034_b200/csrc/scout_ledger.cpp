@@ -178,4 +178,14 @@ int scout_peer_group(const scout_mesh_t *shape, uint64_t rank, uint64_t *peers, 
     return g > cap ? SCOUT_ERR_TRUNCATED : SCOUT_OK;
 }
 
+int scout_rotating_slice(uint64_t numel, uint64_t slice_elems, uint64_t step, uint64_t *begin,
+                         uint64_t *count) {
+    if (!begin || !count || numel == 0 || slice_elems == 0) return SCOUT_ERR_INVALID;
+    const uint64_t n_windows = numel / slice_elems + (numel % slice_elems ? 1 : 0);
+    const uint64_t w = step % n_windows;
+    *begin = w * slice_elems;
+    *count = numel - *begin < slice_elems ? numel - *begin : slice_elems;
+    return SCOUT_OK;
+}
+
 }  // extern "C"

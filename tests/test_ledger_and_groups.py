@@ -155,3 +155,44 @@ def test_peer_group_truncation_and_bad_arguments():
         B.scout_mesh_coords((2, 1, 1, 1, 1, 1), 2)
     with pytest.raises(B.ScoutError):
         B.scout_mesh_size((2, 0, 1, 1, 1, 1))
+
+
+def test_rotating_slice_covers_every_element_once_per_rotation():
+    for numel, slice_elems in ((1, 65536), (65536, 65536), (65537, 65536), (1_000_003, 65536), (10, 3)):
+        n_windows = -(-numel // slice_elems)
+        seen = []
+        for step in range(2 * n_windows + 1):
+            got = B.scout_rotating_slice(numel, slice_elems, step)
+            assert got == H.rotating_slice(numel, slice_elems, step)
+            seen.append(got)
+        one_turn = seen[:n_windows]
+        covered = [i for b, n in one_turn for i in range(b, b + n)] if numel < 10**5 else None
+        if covered is not None:
+            assert covered == list(range(numel))          # every element exactly once per rotation
+        assert sum(n for _, n in one_turn) == numel
+        assert seen[n_windows:2 * n_windows] == one_turn and seen[2 * n_windows] == seen[0]
+    with pytest.raises(B.ScoutError):
+        B.scout_rotating_slice(0, 65536, 0)
+
+
+@pytest.mark.gpu
+def test_signing_a_rotating_slice_localises_a_fault_inside_it():
+    import torch
+    import helpers
+    from paper_2608_11034_b200 import inputs
+    numel, slice_elems = 300_000, 65536
+    spec = inputs.TensorSpec("param", (numel,), "f32", "normal", 0.02)
+    w = inputs.Workload("slice", 0, "x", 3, 16384, [spec], 31)
+    w.patches = [inputs.Patch(2, 0, 200_000, "xor", 1 << 13)]
+    _, views = inputs.generate(w, "cuda")
+    hits = {}
+    for step in range(5):
+        begin, count = B.scout_rotating_slice(numel, slice_elems, step)
+        sw = inputs.Workload("slice", 0, "x", 3, 16384,
+                             [inputs.TensorSpec("param", (count,), "f32", "normal", 0.02)], 31)
+        sviews = [[views[r][0][begin:begin + count]] for r in range(3)]
+        got = helpers.gpu_sign_vote(sw, sviews)
+        hits[step] = got["outliers"]
+    window = 200_000 // slice_elems
+    chunk = (200_000 - window * slice_elems) * 4 // 16384
+    assert hits == {0: [], 1: [], 2: [], 3: [(chunk, 2)], 4: []}
