@@ -242,11 +242,14 @@ SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/)
 
 /* Knobs of a plan (optional).
  *   set "tile_bytes"  bytes per work item, a power of two in [2048, 65536]
- *   set "variant"     scan kernel: 0 = direct 16-byte loads; 1 = the same with the
- *                     next rows prefetched into registers; 2 = bulk-async copies
- *                     (cp.async.bulk + mbarrier) through a per-warp ring in
- *                     shared memory; 3 = read-only probe (measures the memory
- *                     system only: the records it leaves are NOT signatures)
+ *   set "variant"     scan kernel: 0 = direct 16-byte loads (default); 1 = the same
+ *                     with the next rows prefetched into registers; 2 = bulk-async
+ *                     copies (cp.async.bulk + mbarrier) through a per-warp ring in
+ *                     shared memory; 4 = block-wide ring: a producer warp fetches
+ *                     whole tiles (<= 32 KiB) with one bulk copy each and eight
+ *                     consumer warps share them (needs tile_bytes <= 32768);
+ *                     3 = read-only probe (measures the memory system only: the
+ *                     records it leaves are NOT signatures)
  *   set "grid"        CTAs of the scan kernel
  *   set "timing"      1: record CUDA events around the scan kernel on the
  *                     caller's stream

@@ -553,6 +553,7 @@ int scout_plan_set(scout_plan_t *p, const char *key, int64_t value) {
     if (!std::strcmp(key, "tile_bytes")) {
         if (value < 2048 || value > 65536 || (value & (value - 1))) return SCOUT_ERR_INVALID;
         if ((uint32_t)value == p->tile_bytes) return SCOUT_OK;
+        if (p->variant == 4 && value > 32768) return SCOUT_ERR_INVALID;
         p->tile_bytes = (uint32_t)value;
         try {
             build_tiles(p);
@@ -573,7 +574,8 @@ int scout_plan_set(scout_plan_t *p, const char *key, int64_t value) {
         return upload_tables(p);
     }
     if (!std::strcmp(key, "variant")) {
-        if (value < 0 || value > 3) return SCOUT_ERR_INVALID;
+        if (value < 0 || value > 4) return SCOUT_ERR_INVALID;
+        if (value == 4 && p->tile_bytes > 32768) return SCOUT_ERR_INVALID;  // a tile must fit one stage
         p->variant = (int)value;
         return sign_grid_size(p->variant, p->device, &p->grid);
     }

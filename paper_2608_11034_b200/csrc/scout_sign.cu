@@ -268,6 +268,23 @@ struct TileScan {
         fold_row(h, v, m);
         stats_fast<DT>(v, a);
     }
+    // Warp reduction of what the lanes hold: hash share, sums, and whether any lane
+    // suspects a non-finite (or, for bf16, subnormal) element.
+    __device__ __forceinline__ void reduce(uint64_t &h_out, double &s, double &q, bool &suspect) const {
+        q = a.q0 + a.q1;
+        if constexpr (DT == SCOUT_DT_BF16 && BF16_BITROUTE > 0)
+            s = fma(a.s1, 0x1p896, a.s0);  // s1 holds x * 2^-896: exact power-of-two rescale
+        else
+            s = a.s0 + a.s1;
+        suspect = __any_sync(0xFFFFFFFFu, may_hold_nonfinite<DT>(a));
+        h_out = h;
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) {
+            h_out += __shfl_xor_sync(0xFFFFFFFFu, h_out, d);
+            s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
+            q += __shfl_xor_sync(0xFFFFFFFFu, q, d);
+        }
+    }
     // Ragged last row of a chunk (missing words are zero), warp reduction, and the
     // classifying rescan if the tile may hold a non-finite element.
     __device__ __forceinline__ void finish(const uint8_t *tile, uint32_t nbytes, uint32_t lane,
@@ -276,24 +293,16 @@ struct TileScan {
             uint4 v = ld_masked16(tile, (nbytes / ROW_BYTES) * ROW_BYTES + 16u * lane, nbytes);
             row(v);
         }
-        double s, q = a.q0 + a.q1;
-        if constexpr (DT == SCOUT_DT_BF16 && BF16_BITROUTE > 0)
-            s = fma(a.s1, 0x1p896, a.s0);  // s1 holds x * 2^-896: exact power-of-two rescale
-        else
-            s = a.s0 + a.s1;
-        const bool suspect = __any_sync(0xFFFFFFFFu, may_hold_nonfinite<DT>(a));
-#pragma unroll
-        for (int d = 16; d >= 1; d >>= 1) {
-            h += __shfl_xor_sync(0xFFFFFFFFu, h, d);
-            s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
-            q += __shfl_xor_sync(0xFFFFFFFFu, q, d);
-        }
+        double s, q;
+        bool suspect;
+        uint64_t h_tile;
+        reduce(h_tile, s, q, suspect);
         uint32_t nan_count = 0, inf_count = 0;
         if constexpr (DT == SCOUT_DT_F32 || DT == SCOUT_DT_BF16 || DT == SCOUT_DT_F16 ||
                       DT == SCOUT_DT_F64) {
             if (suspect) rescan_classifying<DT>(tile, nbytes, lane, s, q, nan_count, inf_count);
         }
-        out.h = h;
+        out.h = h_tile;
         out.sum = s;
         out.sumsq = q;
         out.nan_count = nan_count;
@@ -647,6 +656,246 @@ __global__ void __launch_bounds__(SIGN_THREADS, SCOUT_RING_BLOCKS) sign_tiles_ri
     }
 }
 
+// ---- front end 4: block-wide bulk-async ring --------------------------------------
+// One CTA = 8 consumer warps + 1 producer warp.  The producer's lane 0 walks the
+// CTA's tiles and fetches each WHOLE tile (<= 32 KiB of whole rows) with one
+// cp.async.bulk into one of CTA_STAGES shared-memory stages, after the stage's
+// "empty" mbarrier says all eight consumers are done with its previous tile.  The
+// consumers wait on the stage's "full" mbarrier; warp w folds rows [8w, 8w+8) of
+// the tile; every lane weights its hash share by the rows that follow its warp's
+// block and leaves (h, sum, sumsq) in shared memory; the last warp to finish a tile
+// (an atomic ticket in shared memory, nobody waits) adds the eight warps' shares
+// lane by lane in warp order, runs the one butterfly of the tile and writes the
+// record.  Large copies keep the copy engine efficient and the bytes
+// in flight (CTA_STAGES x 32 KiB per CTA, 2 CTAs per SM) do not depend on the
+// arithmetic.  Every wait is bounded; a wait that gives up sets the error flag.
+constexpr int CTA_STAGE_BYTES = 32768;
+constexpr int CTA_STAGES = 3;
+constexpr int CTA_CONSUMERS = 8;
+constexpr int CTA_THREADS = (CTA_CONSUMERS + 1) * 32;
+constexpr int CTA_ROWS_PER_WARP = CTA_STAGE_BYTES / (int)ROW_BYTES / CTA_CONSUMERS;  // 8
+
+struct CtaStageInfo {      // written by the producer before the copy, read after the full barrier
+    const uint8_t *tile;
+    TileRec *rec;
+    uint32_t nbytes, dtype;
+};
+// One consumer LANE's part of a tile (no per-warp reduction).  The shares are kept
+// in the stage itself: once warp w has folded its rows, the first kilobyte of its
+// own 4 KiB block (which no other warp reads) holds its 32 lanes' shares.
+struct CtaShare {
+    uint64_t h;
+    double s, q;
+    uint64_t pad;
+};
+static_assert(sizeof(CtaShare) * 32 <= CTA_ROWS_PER_WARP * ROW_BYTES, "shares fit the warp's block");
+struct CtaShared {
+    unsigned long long full[CTA_STAGES], empty[CTA_STAGES];
+    CtaStageInfo info[CTA_STAGES];
+    uint64_t weight[CTA_CONSUMERS];  // P^(rows after warp w's block) in a full tile
+    uint32_t suspect[CTA_STAGES];
+    uint32_t ticket[CTA_STAGES];
+    uint32_t abort_flag;
+};
+constexpr int CTA_SMEM = CTA_STAGES * CTA_STAGE_BYTES + (int)sizeof(CtaShared);
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    uint32_t polls = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if (++polls > RING_WAIT_LIMIT) return false;
+    }
+    return true;
+}
+
+template <int DT>
+__device__ __forceinline__ void cta_consume(const CtaStageInfo &info, uint32_t data, uint32_t warp,
+                                            uint32_t lane, uint64_t weight, CtaShare &out, bool &suspect) {
+    TileScan<DT> st;
+    st.begin(lane);
+    const uint32_t full_rows = info.nbytes / ROW_BYTES;
+    const uint32_t total_rows = (info.nbytes + ROW_BYTES - 1) / ROW_BYTES;
+    const uint32_t row0 = warp * CTA_ROWS_PER_WARP;
+    const uint32_t row1 = min(row0 + CTA_ROWS_PER_WARP, total_rows);
+    const uint32_t saddr = data + row0 * ROW_BYTES + 16u * lane;
+    if (row0 + CTA_ROWS_PER_WARP <= full_rows) {
+        uint4 v[CTA_ROWS_PER_WARP];
+#pragma unroll
+        for (int r = 0; r < CTA_ROWS_PER_WARP; ++r) v[r] = lds16(saddr + r * ROW_BYTES);
+#pragma unroll
+        for (int r = 0; r < CTA_ROWS_PER_WARP; ++r) st.row(v[r]);
+    } else {
+        for (uint32_t r = row0; r < row1; ++r) {
+            if (r < full_rows) st.row(lds16(data + r * ROW_BYTES + 16u * lane));
+            else st.row(ld_masked16(info.tile, r * ROW_BYTES + 16u * lane, info.nbytes));  // ragged row
+        }
+    }
+    // the warp's rows are followed by (total_rows - row1) rows of the tile
+    uint64_t h = st.h;
+    if (row1 > row0) h *= total_rows == (uint32_t)(CTA_STAGE_BYTES / ROW_BYTES) ? weight : pow_p(total_rows - row1);
+    out.h = h;
+    out.q = st.a.q0 + st.a.q1;
+    if constexpr (DT == SCOUT_DT_BF16 && BF16_BITROUTE > 0) out.s = fma(st.a.s1, 0x1p896, st.a.s0);
+    else out.s = st.a.s0 + st.a.s1;
+    suspect = may_hold_nonfinite<DT>(st.a);
+}
+
+template <int DT>
+__device__ __forceinline__ void cta_rescan(const CtaStageInfo &info, uint32_t lane, TileRec &rec) {
+    if constexpr (DT == SCOUT_DT_F32 || DT == SCOUT_DT_BF16 || DT == SCOUT_DT_F16 || DT == SCOUT_DT_F64)
+        rescan_classifying<DT>(info.tile, info.nbytes, lane, rec.sum, rec.sumsq, rec.nan_count, rec.inf_count);
+}
+
+__global__ void __launch_bounds__(CTA_THREADS, 2) sign_tiles_cta_ring(const SignArgs a) {
+    extern __shared__ __align__(128) uint8_t cta_smem[];
+    CtaShared &sh = *reinterpret_cast<CtaShared *>(cta_smem + CTA_STAGES * CTA_STAGE_BYTES);
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const uint64_t n_items = a.n_tiles * a.n_replicas;
+    const uint32_t data0 = smem_u32(cta_smem);
+    pdl_launch_dependents();
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < CTA_STAGES; ++s) {
+            mbar_init(smem_u32(&sh.full[s]), 1);
+            mbar_init(smem_u32(&sh.empty[s]), CTA_CONSUMERS);
+            sh.ticket[s] = 0;
+            sh.suspect[s] = 0;
+        }
+        for (int w = 0; w < CTA_CONSUMERS; ++w)
+            sh.weight[w] = pow_p((uint64_t)CTA_ROWS_PER_WARP * (CTA_CONSUMERS - 1 - w));
+        sh.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == CTA_CONSUMERS) {
+        // ---- producer ----
+        if (lane == 0) {
+            uint32_t n = 0;
+            for (uint64_t item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
+                const uint32_t stage = n % CTA_STAGES;
+                // wait until the consumers have released this stage's previous tile
+                // (the first CTA_STAGES uses find the barrier's "previous" phase complete)
+                if (!mbar_wait_bounded(smem_u32(&sh.empty[stage]), ((n / CTA_STAGES) & 1u) ^ 1u) ||
+                    *(volatile uint32_t *)&sh.abort_flag) {
+                    atomicExch(&sh.abort_flag, 1u);
+                    if (a.error) atomicExch(a.error, 1u);
+                    break;
+                }
+                const uint32_t rr = (uint32_t)(item / a.n_tiles);
+                const uint64_t t = a.tile_begin + (item - (uint64_t)rr * a.n_tiles);
+                const uint32_t r = a.replica_begin + rr;
+                const TileDesc td = a.tiles[t];
+                CtaStageInfo info;
+                info.tile = tile_address(a, td, r);
+                info.rec = &a.recs[(uint64_t)r * a.tiles_per_replica + t];
+                info.nbytes = td.nbytes;
+                info.dtype = td.dtype;
+                sh.info[stage] = info;
+                const uint32_t bytes = (td.nbytes / ROW_BYTES) * ROW_BYTES;
+                const uint32_t bar = smem_u32(&sh.full[stage]);
+                if (bytes) {
+                    mbar_expect_tx(bar, bytes);
+                    bulk_g2s(data0 + stage * CTA_STAGE_BYTES, info.tile, bytes, bar);
+                } else {
+                    mbar_arrive(bar);  // a tile shorter than one row: nothing to copy
+                }
+            }
+        }
+        return;
+    }
+
+    // ---- consumers ----
+    uint32_t n = 0;
+    for (uint64_t item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
+        const uint32_t stage = n % CTA_STAGES;
+        if (!mbar_wait_bounded(smem_u32(&sh.full[stage]), (n / CTA_STAGES) & 1u) ||
+            *(volatile uint32_t *)&sh.abort_flag) {
+            if (lane == 0) {
+                atomicExch(&sh.abort_flag, 1u);
+                if (a.error) atomicExch(a.error, 1u);
+            }
+            break;  // copies already issued are awaited below, before shared memory is released
+        }
+        const CtaStageInfo info = sh.info[stage];
+        const uint32_t data = data0 + stage * CTA_STAGE_BYTES;
+        CtaShare mine;
+        bool sus = false;
+        const uint64_t wgt = sh.weight[warp];
+        switch (info.dtype) {
+            case SCOUT_DT_F32:  cta_consume<SCOUT_DT_F32>(info, data, warp, lane, wgt, mine, sus); break;
+            case SCOUT_DT_BF16: cta_consume<SCOUT_DT_BF16>(info, data, warp, lane, wgt, mine, sus); break;
+            case SCOUT_DT_I64:  cta_consume<SCOUT_DT_I64>(info, data, warp, lane, wgt, mine, sus); break;
+            case SCOUT_DT_F16:  cta_consume<SCOUT_DT_F16>(info, data, warp, lane, wgt, mine, sus); break;
+            case SCOUT_DT_F64:  cta_consume<SCOUT_DT_F64>(info, data, warp, lane, wgt, mine, sus); break;
+            case SCOUT_DT_I32:  cta_consume<SCOUT_DT_I32>(info, data, warp, lane, wgt, mine, sus); break;
+            default:            cta_consume<SCOUT_DT_U8>(info, data, warp, lane, wgt, mine, sus); break;
+        }
+        CtaShare *shares = reinterpret_cast<CtaShare *>(cta_smem + stage * CTA_STAGE_BYTES);
+        __syncwarp();  // every lane of this warp has read its rows: the block may be reused
+        shares[warp * (CTA_ROWS_PER_WARP * ROW_BYTES / sizeof(CtaShare)) + lane] = mine;
+        if (__any_sync(0xFFFFFFFFu, sus) && lane == 0) atomicOr(&sh.suspect[stage], 1u);
+        uint32_t last = 0;
+        __syncwarp();
+        if (lane == 0) {
+            __threadfence_block();
+            last = atomicAdd(&sh.ticket[stage], 1u) == CTA_CONSUMERS - 1;
+        }
+        last = __shfl_sync(0xFFFFFFFFu, last, 0);
+        if (last) {  // every share of this tile is in shared memory: add them in warp order
+            __threadfence_block();
+            uint64_t h = 0;
+            double sum = 0.0, sumsq = 0.0;
+            for (int w = 0; w < CTA_CONSUMERS; ++w) {
+                const volatile CtaShare &x = shares[w * (CTA_ROWS_PER_WARP * ROW_BYTES / sizeof(CtaShare)) + lane];
+                h += x.h;
+                sum += x.s;
+                sumsq += x.q;
+            }
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) {
+                h += __shfl_xor_sync(0xFFFFFFFFu, h, d);
+                sum += __shfl_xor_sync(0xFFFFFFFFu, sum, d);
+                sumsq += __shfl_xor_sync(0xFFFFFFFFu, sumsq, d);
+            }
+            TileRec rec;
+            rec.h = h;
+            rec.sum = sum;
+            rec.sumsq = sumsq;
+            rec.nan_count = rec.inf_count = 0;
+            const uint32_t suspect = *(volatile uint32_t *)&sh.suspect[stage];
+            if (suspect) {
+                switch (info.dtype) {
+                    case SCOUT_DT_F32:  cta_rescan<SCOUT_DT_F32>(info, lane, rec); break;
+                    case SCOUT_DT_BF16: cta_rescan<SCOUT_DT_BF16>(info, lane, rec); break;
+                    case SCOUT_DT_F16:  cta_rescan<SCOUT_DT_F16>(info, lane, rec); break;
+                    case SCOUT_DT_F64:  cta_rescan<SCOUT_DT_F64>(info, lane, rec); break;
+                    default: break;
+                }
+            }
+            if (lane == 0) {
+                store_record(info.rec, rec);
+                sh.ticket[stage] = 0;
+                sh.suspect[stage] = 0;
+            }
+        }
+        __syncwarp();
+        if (lane == 0) {
+            // the shares were written with ordinary stores; order them before the next bulk copy
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mbar_arrive(smem_u32(&sh.empty[stage]));  // this warp is done with the stage
+        }
+    }
+    if (*(volatile uint32_t *)&sh.abort_flag) {
+        // give copies that may still be in flight a bounded chance to land before exit
+        for (int s = 0; s < CTA_STAGES; ++s)
+            for (uint32_t par = 0; par < 2; ++par) mbar_wait_bounded(smem_u32(&sh.full[s]), par);
+    }
+}
+
 // Read-only probe: the same tiles and the same loads as the direct scan, with an
 // XOR as the only arithmetic.  It measures what the memory system delivers to
 // this access pattern (the ceiling the scan is compared with).
@@ -759,7 +1008,10 @@ __global__ void __launch_bounds__(FIN_THREADS) finalize_chunks(const ChunkDesc *
 int sign_grid_size(int variant, int device, int *grid) {
     int sms = 0, per_sm = 0;
     SCOUT_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
-    if (variant == 2) {
+    if (variant == 4) {
+        SCOUT_CUDA(cudaFuncSetAttribute(sign_tiles_cta_ring, cudaFuncAttributeMaxDynamicSharedMemorySize, CTA_SMEM));
+        SCOUT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sign_tiles_cta_ring, CTA_THREADS, CTA_SMEM));
+    } else if (variant == 2) {
         SCOUT_CUDA(cudaFuncSetAttribute(sign_tiles_ring, cudaFuncAttributeMaxDynamicSharedMemorySize, RING_SMEM));
         SCOUT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sign_tiles_ring, SIGN_THREADS, RING_SMEM));
     } else if (variant == 1) {
@@ -791,6 +1043,13 @@ int launch_sign_tiles(const SignLaunch &l, cudaStream_t stream) {
     const uint64_t want = (items + SIGN_THREADS / 32 - 1) / (SIGN_THREADS / 32);
     int grid = l.grid;
     if ((uint64_t)grid > want) grid = (int)want;
+    if (l.variant == 4) {  // one CTA per tile at a time
+        int g = l.grid;
+        if ((uint64_t)g > items) g = (int)items;
+        sign_tiles_cta_ring<<<g, CTA_THREADS, CTA_SMEM, stream>>>(a);
+        SCOUT_CUDA(cudaGetLastError());
+        return SCOUT_OK;
+    }
     switch (l.variant) {
         case 3: read_probe<<<grid, SIGN_THREADS, 0, stream>>>(a); break;
         case 2: sign_tiles_ring<<<grid, SIGN_THREADS, RING_SMEM, stream>>>(a); break;
