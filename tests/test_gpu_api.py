@@ -1,0 +1,102 @@
+"""Behaviour of the C ABI beyond the main path: plan knobs, re-binding, user
+streams, host-resident replicas in pageable and scattered memory."""
+import numpy as np
+import pytest
+import torch
+
+import helpers
+from oracle import scout_oracle as orc
+from paper_2608_11034_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def test_plan_knobs():
+    from paper_2608_11034_b200 import binding as B
+    w = inputs.workload(1, "default", 1 / 8)
+    _, views = inputs.generate(w, "cuda")
+    plan = helpers.gpu_plan(w)
+    h = plan.handle
+    assert B.scout_plan_get(h, "tile_bytes") in (4096, 8192, 16384, 32768)
+    assert B.scout_plan_get(h, "variant") == 0 and B.scout_plan_get(h, "grid") > 0
+    n0 = B.scout_plan_get(h, "n_tiles")
+    B.scout_plan_set(h, "tile_bytes", 2048)
+    assert B.scout_plan_get(h, "n_tiles") == w.bytes_per_replica // 2048 != n0
+    assert B.scout_plan_get(h, "scratch_bytes") == B.scout_plan_get(h, "n_tiles") * w.R * 32
+    for key, bad in (("tile_bytes", 1000), ("tile_bytes", 131072), ("variant", 5), ("variant", -1),
+                     ("grid", 0), ("nonsense", 1)):
+        with pytest.raises(B.ScoutError):
+            B.scout_plan_set(h, key, bad)
+    with pytest.raises(B.ScoutError):
+        B.scout_plan_get(h, "nonsense")
+    with pytest.raises(B.ScoutError):            # timing was never switched on
+        B.scout_plan_get(h, "last_sign_ns")
+    B.scout_plan_set(h, "tile_bytes", 65536)
+    with pytest.raises(B.ScoutError):            # the block-wide ring needs a tile that fits one stage
+        B.scout_plan_set(h, "variant", 4)
+    B.scout_plan_set(h, "tile_bytes", 8192)
+    B.scout_plan_set(h, "grid", 7)               # a tiny grid must still give the same records
+    B.scout_plan_set(h, "timing", 1)
+    plan.bind(views)
+    plan.sign_and_vote()
+    got = plan.fetch()
+    assert B.scout_plan_get(h, "last_sign_ns") > 0 and B.scout_plan_get(h, "device_error") == 0
+    ref = helpers.gpu_sign_vote(w, views)
+    assert (got["sigs"]["hash"] == ref["sigs"]["hash"]).all() and got["outliers"] == ref["outliers"]
+    plan.close()
+
+
+def test_rebinding_and_user_streams():
+    from paper_2608_11034_b200 import binding as B
+    w = inputs.workload(2, "mantissa", 1 / 64)
+    _, views_a = inputs.generate(w, "cuda")
+    wb = inputs.workload(2, "clean", 1 / 64)
+    wb.seed += 100
+    _, views_b = inputs.generate(wb, "cuda")
+    plan = helpers.gpu_plan(w)
+    side = torch.cuda.Stream()
+    results = []
+    for views in (views_a, views_b, views_a):
+        plan.bind(views)
+        with torch.cuda.stream(side):
+            plan.sign_and_vote()            # enqueued on the side stream (the current one)
+            side.synchronize()
+        results.append(plan.fetch())
+    assert len(results[0]["outliers"]) == 1 and results[1]["outliers"] == []
+    assert results[0]["sigs"].tobytes() == results[2]["sigs"].tobytes()
+    assert (results[0]["sigs"]["hash"] != results[1]["sigs"]["hash"]).all()
+    rep = plan.certify(stream=side.cuda_stream)
+    assert rep["outliers"] == results[0]["outliers"]
+    plan.close()
+
+
+def test_certify_host_with_pageable_and_scattered_tensors():
+    from paper_2608_11034_b200 import binding as B
+    w = inputs.workload(5, "default", 1 / 400)
+    _, views = inputs.generate(w, "cpu")
+    osigs, _ = helpers.oracle_sign_all(w, views)
+    want = orc.certify(osigs)
+    # every tensor in its own pageable allocation, replicas interleaved: nothing is contiguous
+    keep = [[v.clone() for v in rep] for rep in views]
+    ptrs = [t.data_ptr() for rep in keep for t in rep]
+    plan = helpers.gpu_plan(w)
+    got = B.scout_certify_host(plan.handle, ptrs)
+    assert got["report"] == want["report"] and got["outliers"] == want["outliers"]
+    # change the tiling after the staging buffers exist, then run again from flat pinned buffers
+    B.scout_plan_set(plan.handle, "tile_bytes", 4096)
+    flats = []
+    for rep in views:
+        offs, total = inputs.packed_offsets(w.specs)
+        f = torch.zeros(total, dtype=torch.uint8).pin_memory()
+        for o, v in zip(offs, rep):
+            f[o:o + v.numel() * v.element_size()] = v.view(-1).view(torch.uint8)
+        flats.append(f)
+    fviews = [inputs.tensor_views(f, w.specs) for f in flats]
+    got2 = B.scout_certify_host(plan.handle, [v.data_ptr() for rep in fviews for v in rep])
+    assert got2["report"] == want["report"] and got2["outliers"] == want["outliers"]
+    # device-resident certify on the same plan still works after the host runs
+    dviews = [[v.cuda() for v in rep] for rep in views]
+    plan.bind(dviews)
+    got3 = plan.certify()
+    assert got3["report"] == want["report"]
+    plan.close()
