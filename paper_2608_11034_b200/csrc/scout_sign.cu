@@ -940,6 +940,54 @@ __global__ void __launch_bounds__(SIGN_THREADS) read_probe(const SignArgs a) {
 // per lane in ascending tile order and then through a fixed butterfly.
 constexpr int FIN_THREADS = 128;
 
+// One warp turns the tile records of one (chunk, replica) into its signature record
+// (valid in lane 0).  tr: the chunk's nt records in order; every tile but the last
+// has tile_rows rows; p_stride = P^(32 * tile_rows).
+__device__ __forceinline__ scout_sig_t combine_tiles(const TileRec *tr, uint32_t nt, uint64_t nbytes,
+                                                     uint64_t k, uint32_t dtype, uint64_t meta,
+                                                     uint32_t tile_rows, uint64_t p_stride, uint32_t lane) {
+    const uint64_t rows_total = (nbytes + ROW_BYTES - 1) / ROW_BYTES;
+    const uint64_t rows_last = rows_total - (uint64_t)(nt - 1) * tile_rows;
+    uint64_t h = 0;
+    double s = 0.0, q = 0.0;
+    uint32_t nan_count = 0, inf_count = 0, last_t = 0;
+    const uint32_t n_full = nt - 1;  // every tile but the chunk's last has tile_rows rows
+    for (uint32_t t = lane; t < n_full; t += 32) {
+        const TileRec x = tr[t];
+        h = h * p_stride + x.h;
+        s += x.sum;
+        q += x.sumsq;
+        nan_count += x.nan_count;
+        inf_count += x.inf_count;
+        last_t = t;
+    }
+    if (lane < n_full) h *= pow_p(rows_last + (uint64_t)tile_rows * (n_full - 1 - last_t));
+    if (lane == (n_full & 31u)) {  // the last (possibly short) tile: nothing follows it
+        const TileRec x = tr[n_full];
+        h += x.h;
+        s += x.sum;
+        q += x.sumsq;
+        nan_count += x.nan_count;
+        inf_count += x.inf_count;
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        h += __shfl_xor_sync(0xFFFFFFFFu, h, d);
+        s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
+        q += __shfl_xor_sync(0xFFFFFFFFu, q, d);
+        nan_count += __shfl_xor_sync(0xFFFFFFFFu, nan_count, d);
+        inf_count += __shfl_xor_sync(0xFFFFFFFFu, inf_count, d);
+    }
+    scout_sig_t o;
+    o.hash = finalize_hash(h, nbytes, k, dtype, meta);
+    o.nan_count = nan_count;
+    o.inf_count = inf_count;
+    o.sum = s;
+    o.sumsq = q;
+    return o;
+}
+
+
 __global__ void __launch_bounds__(FIN_THREADS) finalize_chunks(const ChunkDesc *chunks, uint64_t C,
                                                                uint32_t R, const TileRec *recs,
                                                                uint64_t tiles_per_replica,
@@ -956,48 +1004,9 @@ __global__ void __launch_bounds__(FIN_THREADS) finalize_chunks(const ChunkDesc *
         const uint64_t c = item / R;
         const uint32_t r = (uint32_t)(item - c * R);
         const ChunkDesc cd = chunks[c];
-        const TileRec *tr = recs + (uint64_t)r * tiles_per_replica + cd.tile0;
-        const uint32_t nt = cd.ntiles;
-        const uint64_t rows_total = (cd.nbytes + ROW_BYTES - 1) / ROW_BYTES;
-        const uint64_t rows_last = rows_total - (uint64_t)(nt - 1) * tile_rows;
-
-        uint64_t h = 0;
-        double s = 0.0, q = 0.0;
-        uint32_t nan_count = 0, inf_count = 0, last_t = 0;
-        const uint32_t n_full = nt - 1;  // every tile but the chunk's last has tile_rows rows
-        for (uint32_t t = lane; t < n_full; t += 32) {
-            const TileRec x = tr[t];
-            h = h * p_stride + x.h;
-            s += x.sum;
-            q += x.sumsq;
-            nan_count += x.nan_count;
-            inf_count += x.inf_count;
-            last_t = t;
-        }
-        if (lane < n_full) h *= pow_p(rows_last + (uint64_t)tile_rows * (n_full - 1 - last_t));
-        if (lane == (n_full & 31u)) {  // the last (possibly short) tile: nothing follows it
-            const TileRec x = tr[n_full];
-            h += x.h;
-            s += x.sum;
-            q += x.sumsq;
-            nan_count += x.nan_count;
-            inf_count += x.inf_count;
-        }
-#pragma unroll
-        for (int d = 16; d >= 1; d >>= 1) {
-            h += __shfl_xor_sync(0xFFFFFFFFu, h, d);
-            s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
-            q += __shfl_xor_sync(0xFFFFFFFFu, q, d);
-            nan_count += __shfl_xor_sync(0xFFFFFFFFu, nan_count, d);
-            inf_count += __shfl_xor_sync(0xFFFFFFFFu, inf_count, d);
-        }
+        const scout_sig_t o = combine_tiles(recs + (uint64_t)r * tiles_per_replica + cd.tile0, cd.ntiles,
+                                            cd.nbytes, cd.k, cd.dtype, cd.meta, tile_rows, p_stride, lane);
         if (lane == 0) {
-            scout_sig_t o;
-            o.hash = finalize_hash(h, cd.nbytes, cd.k, cd.dtype, cd.meta);
-            o.nan_count = nan_count;
-            o.inf_count = inf_count;
-            o.sum = s;
-            o.sumsq = q;
             sigs[c * R + r] = o;
         }
     }
@@ -1128,8 +1137,7 @@ __global__ void __launch_bounds__(SIGN_THREADS) sign_tiles_noalloc(const __grid_
     }
 }
 
-// Same combine as finalize_chunks (segment identity over tiles, fixed order for
-// the fp64 partials), for a single tensor whose chunk geometry is arithmetic.
+// The combine of finalize_chunks for a single tensor whose chunk geometry is arithmetic.
 __global__ void __launch_bounds__(FIN_THREADS) finalize_noalloc(const __grid_constant__ NoallocArgs a,
                                                                 uint64_t C, uint64_t p_stride) {
     const uint32_t lane = threadIdx.x & 31u;
@@ -1141,46 +1149,9 @@ __global__ void __launch_bounds__(FIN_THREADS) finalize_noalloc(const __grid_con
         const uint32_t r = (uint32_t)(item - c * a.R);
         const uint64_t chunk_n = min(a.chunk_bytes, a.nbytes - c * a.chunk_bytes);
         const uint32_t nt = (uint32_t)((chunk_n + a.tile_bytes - 1) / a.tile_bytes);
-        const TileRec *tr = a.recs + (uint64_t)r * a.n_tiles + c * a.tiles_per_chunk;
-        const uint64_t rows_total = (chunk_n + ROW_BYTES - 1) / ROW_BYTES;
-        const uint64_t rows_last = rows_total - (uint64_t)(nt - 1) * tile_rows;
-        uint64_t h = 0;
-        double s = 0.0, q = 0.0;
-        uint32_t nan_count = 0, inf_count = 0, last_t = 0;
-        const uint32_t n_full = nt - 1;
-        for (uint32_t t = lane; t < n_full; t += 32) {
-            const TileRec x = tr[t];
-            h = h * p_stride + x.h;
-            s += x.sum;
-            q += x.sumsq;
-            nan_count += x.nan_count;
-            inf_count += x.inf_count;
-            last_t = t;
-        }
-        if (lane < n_full) h *= pow_p(rows_last + (uint64_t)tile_rows * (n_full - 1 - last_t));
-        if (lane == (n_full & 31u)) {
-            const TileRec x = tr[n_full];
-            h += x.h;
-            s += x.sum;
-            q += x.sumsq;
-            nan_count += x.nan_count;
-            inf_count += x.inf_count;
-        }
-#pragma unroll
-        for (int d = 16; d >= 1; d >>= 1) {
-            h += __shfl_xor_sync(0xFFFFFFFFu, h, d);
-            s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
-            q += __shfl_xor_sync(0xFFFFFFFFu, q, d);
-            nan_count += __shfl_xor_sync(0xFFFFFFFFu, nan_count, d);
-            inf_count += __shfl_xor_sync(0xFFFFFFFFu, inf_count, d);
-        }
+        const scout_sig_t o = combine_tiles(a.recs + (uint64_t)r * a.n_tiles + c * a.tiles_per_chunk, nt,
+                                            chunk_n, c, a.dtype, a.meta, tile_rows, p_stride, lane);
         if (lane == 0) {
-            scout_sig_t o;
-            o.hash = finalize_hash(h, chunk_n, c, a.dtype, a.meta);
-            o.nan_count = nan_count;
-            o.inf_count = inf_count;
-            o.sum = s;
-            o.sumsq = q;
             a.sigs[c * a.R + r] = o;
         }
     }
