@@ -52,10 +52,17 @@ def lib():
     """Load the C-ABI library; raise loudly if it is missing (no CPU fallback)."""
     global _lib
     if _lib is None:
+        if not os.path.exists(LIB_PATH) and not os.environ.get("SCOUT_LIB"):
+            try:                      # a source checkout: compile the library once, in-tree
+                from . import build as _build
+                _build.build()
+            except Exception as e:    # noqa: BLE001
+                raise RuntimeError(
+                    f"{LIB_PATH} is missing and could not be built ({e!r}): run "
+                    "`python -m paper_2608_11034_b200.build` (needs nvcc); this package has no "
+                    "CPU fallback") from e
         if not os.path.exists(LIB_PATH):
-            raise RuntimeError(
-                f"{LIB_PATH} is missing: build it with `python -m paper_2608_11034_b200.build` "
-                "(needs nvcc); this package has no CPU fallback")
+            raise RuntimeError(f"{LIB_PATH} is missing; this package has no CPU fallback")
         L = C.CDLL(LIB_PATH)
         vp, u64, u32, i64 = C.c_void_p, C.c_uint64, C.c_uint32, C.c_int64
         sigs = {
