@@ -26,6 +26,13 @@ namespace scout {
 namespace {
 
 constexpr int SIGN_THREADS = 256;
+// Compile-time settings (the defaults are the measured optimum on B200; build.py
+// can compile a copy with others, selected at run time by the SCOUT_LIB variable):
+//   SCOUT_UNROLL         rows (16 B per lane each) a warp has in flight, direct scan
+//   SCOUT_MINBLOCKS      CTAs per SM the direct scan is compiled for (caps registers)
+//   SCOUT_MINBLOCKS_PF   the same for the register-prefetch front end
+//   SCOUT_BF16_BITROUTE  see below
+//   SCOUT_RING_PIECE / _STAGES / _BLOCKS   geometry of the per-warp bulk-async ring
 #ifndef SCOUT_MINBLOCKS
 #define SCOUT_MINBLOCKS 4
 #endif
