@@ -262,6 +262,13 @@ SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/)
 SCOUT_API int scout_plan_set(scout_plan_t *plan, const char *key, int64_t value);
 SCOUT_API int scout_plan_get(const scout_plan_t *plan, const char *key, int64_t *value);
 
+/* Diagnostic: the bulk-async scan kernels wait for their copies with a time limit
+ * (2 s) and report through "device_error" instead of hanging.  This call runs that
+ * wait on a barrier nothing ever signals, with the given limit (<= 1 s):
+ * d_out (device, 2 words) receives {1 if the wait gave up, nanoseconds waited}.
+ * The kernel returns normally and the context stays usable.  Asynchronous. */
+SCOUT_API int scout_selftest_bounded_wait(uint64_t limit_ns, uint64_t *d_out /*device [2]*/, void *stream);
+
 SCOUT_API const char *scout_strerror(int code);
 SCOUT_API int scout_version(void);
 /* Name of the CUDA error behind the calling thread's most recent SCOUT_ERR_CUDA ("" if none). */

@@ -96,6 +96,7 @@ def lib():
             "scout_peer_group": (C.c_int, [vp, u64, vp, u64, C.POINTER(u64), C.POINTER(C.c_int)]),
             "scout_consensus_timing": (C.c_int, [u32, u64, vp, C.c_double, vp, vp, vp, vp, vp]),
             "scout_rotating_slice": (C.c_int, [u64, u64, u64, C.POINTER(u64), C.POINTER(u64)]),
+            "scout_selftest_bounded_wait": (C.c_int, [u64, vp, vp]),
             "scout_strerror": (C.c_char_p, [C.c_int]),
             "scout_version": (C.c_int, []),
             "scout_last_cuda_error": (C.c_char_p, []),
@@ -346,6 +347,10 @@ def scout_rotating_slice(numel: int, slice_elems: int, step: int):
     _check(lib().scout_rotating_slice(numel, slice_elems, step, C.byref(b), C.byref(n)),
            "scout_rotating_slice")
     return b.value, n.value
+
+
+def scout_selftest_bounded_wait(limit_ns: int, d_out: int, stream: int) -> None:
+    _check(lib().scout_selftest_bounded_wait(limit_ns, d_out, stream), "scout_selftest_bounded_wait")
 
 
 def scout_version() -> int:

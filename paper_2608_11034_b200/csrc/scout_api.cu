@@ -618,6 +618,11 @@ int scout_plan_get(const scout_plan_t *p, const char *key, int64_t *value) {
     return SCOUT_OK;
 }
 
+int scout_selftest_bounded_wait(uint64_t limit_ns, uint64_t *d_out, void *stream) {
+    if (!d_out || limit_ns == 0 || limit_ns > 1000000000ull) return SCOUT_ERR_INVALID;
+    return launch_bounded_wait_selftest(limit_ns, d_out, (cudaStream_t)stream);
+}
+
 const char *scout_strerror(int code) {
     switch (code) {
         case SCOUT_OK: return "ok";

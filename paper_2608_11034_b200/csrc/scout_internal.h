@@ -153,6 +153,7 @@ struct SignLaunch {
 };
 int launch_sign_tiles(const SignLaunch &a, cudaStream_t stream);
 int sign_grid_size(int variant, int device, int *grid);
+int launch_bounded_wait_selftest(uint64_t limit_ns, uint64_t *d_out, cudaStream_t stream);
 
 // zero_out (may be null): a CertifyOut the finalise kernel clears for the vote that follows
 int launch_finalize(const ChunkDesc *chunks, uint64_t C, uint32_t R, const TileRec *recs,

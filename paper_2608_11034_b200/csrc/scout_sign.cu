@@ -469,7 +469,7 @@ constexpr int RING_STAGES = SCOUT_RING_STAGES;
 constexpr int RING_ROWS = RING_PIECE / (int)ROW_BYTES;
 constexpr int RING_WARPS = SIGN_THREADS / 32;
 constexpr int RING_SMEM = RING_WARPS * RING_STAGES * RING_PIECE + RING_WARPS * RING_STAGES * 8;
-constexpr uint32_t RING_WAIT_LIMIT = 1u << 24;  // polls before a wait gives up
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // a wait on a copy gives up after 2 s
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
     return (uint32_t)__cvta_generic_to_shared(p);
@@ -490,6 +490,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "r"(bar), "r"(parity)
         : "memory");
     return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Wait for an mbarrier phase, but never longer than limit_ns: the clock is read every
+// 256 polls; false means the wait gave up (the caller reports it and returns).
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
+                                                  unsigned long long limit_ns = WAIT_LIMIT_NS) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t polls = 1;; ++polls) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((polls & 255u) == 0u && global_ns() - t0 > limit_ns) return false;
+    }
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile(
@@ -568,10 +584,7 @@ struct RingCtx {
     __device__ __forceinline__ bool acquire(uint32_t &saddr) {
         const uint32_t stage = consumed % RING_STAGES;
         const uint32_t parity = (consumed / RING_STAGES) & 1u;
-        uint32_t polls = 0;
-        while (!mbar_try_wait(bar0 + 8 * stage, parity)) {
-            if (++polls > RING_WAIT_LIMIT) { gave_up = true; return false; }
-        }
+        if (!mbar_wait_bounded(bar0 + 8 * stage, parity)) { gave_up = true; return false; }
         saddr = data0 + stage * RING_PIECE + 16u * lane;
         return true;
     }
@@ -657,8 +670,7 @@ __global__ void __launch_bounds__(SIGN_THREADS, SCOUT_RING_BLOCKS) sign_tiles_ri
         if (lane == 0 && a.error) atomicExch(a.error, 1u);
         for (uint32_t n = c.consumed; n < c.issued; ++n) {
             const uint32_t stage = n % RING_STAGES, parity = (n / RING_STAGES) & 1u;
-            uint32_t polls = 0;
-            while (!mbar_try_wait(c.bar0 + 8 * stage, parity) && ++polls <= RING_WAIT_LIMIT) {}
+            mbar_wait_bounded(c.bar0 + 8 * stage, parity);
         }
     }
 }
@@ -709,14 +721,6 @@ constexpr int CTA_SMEM = CTA_STAGES * CTA_STAGE_BYTES + (int)sizeof(CtaShared);
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-    uint32_t polls = 0;
-    while (!mbar_try_wait(bar, parity)) {
-        if (++polls > RING_WAIT_LIMIT) return false;
-    }
-    return true;
-}
-
 template <int DT>
 __device__ __forceinline__ void cta_consume(const CtaStageInfo &info, uint32_t data, uint32_t warp,
                                             uint32_t lane, uint64_t weight, CtaShare &out, bool &suspect) {
@@ -903,6 +907,25 @@ __global__ void __launch_bounds__(CTA_THREADS, 2) sign_tiles_cta_ring(const Sign
     }
 }
 
+// Self-test of the bounded wait: an mbarrier that nothing ever arrives on.  The wait
+// must give up after limit_ns and the kernel must return normally; out[0] = 1 if it
+// gave up, out[1] = nanoseconds waited.
+__global__ void bounded_wait_selftest(unsigned long long limit_ns, unsigned long long *out) {
+    __shared__ unsigned long long bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const unsigned long long t0 = global_ns();
+    const bool arrived = mbar_wait_bounded(smem_u32(&bar), 0, limit_ns);
+    const unsigned long long dt = global_ns() - t0;
+    if (threadIdx.x == 0) {
+        out[0] = arrived ? 0ull : 1ull;
+        out[1] = dt;
+    }
+}
+
 // Read-only probe: the same tiles and the same loads as the direct scan, with an
 // XOR as the only arithmetic.  It measures what the memory system delivers to
 // this access pattern (the ceiling the scan is compared with).
@@ -1072,6 +1095,12 @@ int launch_sign_tiles(const SignLaunch &l, cudaStream_t stream) {
         case 1: sign_tiles_direct<1><<<grid, SIGN_THREADS, 0, stream>>>(a); break;
         default: sign_tiles_direct<0><<<grid, SIGN_THREADS, 0, stream>>>(a); break;
     }
+    SCOUT_CUDA(cudaGetLastError());
+    return SCOUT_OK;
+}
+
+int launch_bounded_wait_selftest(uint64_t limit_ns, uint64_t *d_out, cudaStream_t stream) {
+    bounded_wait_selftest<<<1, 32, 0, stream>>>(limit_ns, (unsigned long long *)d_out);
     SCOUT_CUDA(cudaGetLastError());
     return SCOUT_OK;
 }

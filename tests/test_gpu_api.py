@@ -100,3 +100,22 @@ def test_certify_host_with_pageable_and_scattered_tensors():
     got3 = plan.certify()
     assert got3["report"] == want["report"]
     plan.close()
+
+
+def test_a_wait_that_nothing_satisfies_gives_up_and_the_context_survives():
+    """The bulk-async kernels never spin without a limit: a wait on a barrier that is
+    never signalled returns after its time limit with a status the host can read."""
+    from paper_2608_11034_b200 import binding as B
+    out = torch.zeros(2, dtype=torch.int64, device="cuda")
+    limit = 2_000_000                                      # 2 ms
+    B.scout_selftest_bounded_wait(limit, out.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    gave_up, waited = [int(x) for x in out.cpu()]
+    assert gave_up == 1 and limit <= waited < 100 * limit
+    # the context is intact: an ordinary run right after it works
+    w = inputs.workload(1, "default", 1 / 16)
+    _, views = inputs.generate(w, "cuda")
+    got = helpers.gpu_sign_vote(w, views, variant=4)
+    assert len(got["outliers"]) == 1
+    with pytest.raises(B.ScoutError):
+        B.scout_selftest_bounded_wait(0, out.data_ptr(), 0)
