@@ -118,9 +118,15 @@ SCOUT_API int scout_plan_create(uint32_t R, uint64_t T, const scout_tensor_t *te
 
 /* ptrs: host array of R*T device addresses, replica-major (ptrs[r*T + t] is
  * tensor t of replica r), each 16-byte aligned (else SCOUT_ERR_ALIGN) and
- * readable for tensors[t].nbytes.  The table is copied to the device on the
- * default stream; the buffers stay the caller's.  May be called again to scan
- * other buffers of the same geometry. */
+ * readable for tensors[t].nbytes.  The buffers stay the caller's.  May be
+ * called again to scan other buffers of the same geometry: the call first waits
+ * (on the host) until the plan's most recent sign or certify has finished on
+ * whatever stream it was given, so a scan in flight never sees the table change
+ * under it, then copies the table synchronously.
+ *
+ * Every call that takes a plan must be made with the plan's device current (the
+ * device that was current in scout_plan_create); with another device current it
+ * returns SCOUT_ERR_INVALID and launches nothing. */
 SCOUT_API int scout_plan_bind(scout_plan_t *plan, const void *const *ptrs /*host*/);
 
 SCOUT_API int scout_plan_num_chunks(const scout_plan_t *plan, uint64_t *C);
@@ -227,8 +233,11 @@ SCOUT_API int scout_certify_host(scout_plan_t *plan, const void *const *h_ptrs /
  * Limit: R * (number of 64 KiB tiles) <= 65536 records, i.e. about 4 GiB of
  * replica data per call; more returns SCOUT_ERR_UNSUPPORTED and launches
  * nothing.  The first call on each device looks up the array's device address
- * (cudaGetSymbolAddress, with that device current); make that first call
- * before any stream capture.  All calls share the one array and every call
+ * (cudaGetSymbolAddress, with that device current) and is the first launch of
+ * this entry point's two kernels, which makes the CUDA runtime load them; that
+ * loading may itself take device memory.  So make one warm-up call per device
+ * at start-up, while memory is still available and before any stream capture;
+ * the calls after it allocate nothing.  All calls share the one array and every call
  * overwrites the records it reads, so nothing needs clearing between calls,
  * but two calls whose kernels overlap on the GPU (different streams, or several
  * host threads) race on it: serialise them.  Asynchronous on `stream`. */
@@ -255,7 +264,13 @@ SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/)
  *                     caller's stream
  *   get "last_sign_ns" device time of the most recent scan kernel (needs
  *                     "timing" and a synchronised stream)
- *   get "device_error" 1 if a kernel's bounded wait ever gave up (synchronises)
+ *   get "device_error" 1 if a kernel's bounded wait gave up since the flag was last
+ *                     cleared (synchronises); the records of such a run are not
+ *                     valid.  scout_certify and scout_certify_host report it as
+ *                     SCOUT_ERR_CUDA once and clear it; after scout_sign_chunks
+ *                     (asynchronous, so it cannot report) read it here.
+ *   set "device_error" 0 clears the flag; a non-zero value sets it from the host
+ *                     (a way to exercise the error path without a GPU fault)
  *   get "n_tiles", "scratch_bytes", and every settable key
  * Results do not depend on tile_bytes, variant or grid except for the rounding
  * order of the floating-point sums. */

@@ -53,6 +53,7 @@ struct scout_plan {
     std::vector<TileDesc> tiles;
     uint32_t tile_bytes = 0;
     int variant = 0, device = 0, grid = 0;
+    int uniform_dtype = -1;  // dtype of every tensor, or -1 if they differ
     bool bound = false;
 
     TileDesc *d_tiles = nullptr;
@@ -78,12 +79,32 @@ struct scout_plan {
     cudaStream_t s_copy = nullptr, s_comp = nullptr;
     cudaEvent_t ev_copied[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr};
 
+    // recorded after the last kernel of every launch sequence: scout_plan_bind waits for it
+    // before it rewrites the pointer table
+    cudaEvent_t ev_last = nullptr;
+    bool launched = false;
+
     // optional in-stream timing of the scan kernel (key "timing")
     bool timing = false;
     cudaEvent_t ev_t0 = nullptr, ev_t1 = nullptr;
 };
 
 namespace {
+
+// A plan's tables, scratch and events live on the device that was current when it was
+// created; using it with another device current would launch on the wrong GPU.
+int check_device(const scout_plan *p) {
+    int d = -1;
+    SCOUT_CUDA(cudaGetDevice(&d));
+    return d == p->device ? SCOUT_OK : SCOUT_ERR_INVALID;
+}
+
+// Marks the end of a launch sequence on `stream` (see scout_plan_bind).
+int mark_launched(scout_plan *p, cudaStream_t stream) {
+    SCOUT_CUDA(cudaEventRecord(p->ev_last, stream));
+    p->launched = true;
+    return SCOUT_OK;
+}
 
 uint32_t auto_tile_bytes(uint64_t total_bytes) {
     // About two work items per resident warp, 4 KiB .. 32 KiB, power of two (measured:
@@ -143,13 +164,16 @@ int sign_all(scout_plan *p, cudaStream_t stream, scout_sig_t *d_sigs, CertifyOut
     l.recs = p->d_recs;
     l.error = p->d_error;
     l.variant = p->variant;
+    l.uniform_dtype = p->uniform_dtype;
     l.grid = p->grid;
     if (p->timing) SCOUT_CUDA(cudaEventRecord(p->ev_t0, stream));
     int rc = launch_sign_tiles(l, stream);
     if (rc) return rc;
     if (p->timing) SCOUT_CUDA(cudaEventRecord(p->ev_t1, stream));
-    return launch_finalize(p->d_chunks, p->chunks.size(), p->R, p->d_recs, p->tiles.size(),
-                           p->tile_bytes / ROW_BYTES, d_sigs, zero_out, stream);
+    rc = launch_finalize(p->d_chunks, p->chunks.size(), p->R, p->d_recs, p->tiles.size(),
+                         p->tile_bytes / ROW_BYTES, d_sigs, zero_out, stream);
+    if (rc) return rc;
+    return mark_launched(p, stream);
 }
 
 int ensure_certify_buffers(scout_plan *p, uint64_t outlier_cap, uint64_t undecided_cap) {
@@ -234,6 +258,9 @@ int vote_and_report(scout_plan *p, cudaStream_t stream, scout_report_t *report,
                                   : (o.counts[2] ? SCOUT_VERDICT_ATTRIBUTED : SCOUT_CERTIFIED);
     p->have_results = true;
     if (hh->dev_err) {
+        // reported once: the flag is cleared so that the next run starts clean
+        SCOUT_CUDA(cudaMemsetAsync(p->d_error, 0, sizeof(uint32_t), stream));
+        SCOUT_CUDA(cudaStreamSynchronize(stream));
         set_cuda_error(cudaErrorUnknown, "scan kernel: a bounded wait for a bulk copy gave up");
         return SCOUT_ERR_CUDA;
     }
@@ -287,6 +314,9 @@ int scout_plan_create(uint32_t R, uint64_t T, const scout_tensor_t *tensors, uin
                 p->chunks.push_back(cd);
             }
         }
+        p->uniform_dtype = (int)tensors[0].dtype;
+        for (uint64_t t = 1; t < T; ++t)
+            if ((int)tensors[t].dtype != p->uniform_dtype) p->uniform_dtype = -1;
         p->tensor_chunk0[T] = p->chunks.size();
         p->tensor_poff[T] = poff;
         if (p->chunks.size() > 0xFFFFFFFFull) {
@@ -302,7 +332,7 @@ int scout_plan_create(uint32_t R, uint64_t T, const scout_tensor_t *tensors, uin
     int rc = SCOUT_OK;
     do {
         if (cudaGetDevice(&p->device) != cudaSuccess) { rc = SCOUT_ERR_CUDA; break; }
-        if ((rc = sign_grid_size(p->variant, p->device, &p->grid))) break;
+        if ((rc = sign_grid_size(p->variant, p->uniform_dtype, p->device, &p->grid))) break;
         if ((rc = upload_tables(p))) break;
         if (cudaMalloc(&p->d_tensor_chunk0, (T + 1) * sizeof(uint64_t)) != cudaSuccess ||
             cudaMalloc(&p->d_ptrs, (size_t)R * T * sizeof(void *)) != cudaSuccess ||
@@ -310,7 +340,8 @@ int scout_plan_create(uint32_t R, uint64_t T, const scout_tensor_t *tensors, uin
             rc = SCOUT_ERR_NOMEM;
             break;
         }
-        if (cudaMemset(p->d_error, 0, sizeof(uint32_t)) != cudaSuccess) {
+        if (cudaMemset(p->d_error, 0, sizeof(uint32_t)) != cudaSuccess ||
+            cudaEventCreateWithFlags(&p->ev_last, cudaEventDisableTiming) != cudaSuccess) {
             rc = SCOUT_ERR_CUDA;
             break;
         }
@@ -335,6 +366,10 @@ int scout_plan_bind(scout_plan_t *p, const void *const *ptrs) {
         if (!ptrs[i]) return SCOUT_ERR_INVALID;
         if ((uintptr_t)ptrs[i] & 15u) return SCOUT_ERR_ALIGN;
     }
+    int rc = check_device(p);
+    if (rc) return rc;
+    // a scan that is still running reads the table: wait for the plan's last launch first
+    if (p->launched) SCOUT_CUDA(cudaEventSynchronize(p->ev_last));
     SCOUT_CUDA(cudaMemcpy(p->d_ptrs, ptrs, n * sizeof(void *), cudaMemcpyHostToDevice));
     p->bound = true;
     return SCOUT_OK;
@@ -380,6 +415,7 @@ int scout_plan_destroy(scout_plan_t *p) {
     }
     if (p->s_copy) cudaStreamDestroy(p->s_copy);
     if (p->s_comp) cudaStreamDestroy(p->s_comp);
+    if (p->ev_last) cudaEventDestroy(p->ev_last);
     if (p->ev_t0) cudaEventDestroy(p->ev_t0);
     if (p->ev_t1) cudaEventDestroy(p->ev_t1);
     (void)cudaGetLastError();
@@ -390,6 +426,8 @@ int scout_plan_destroy(scout_plan_t *p) {
 int scout_sign_chunks(scout_plan_t *p, void *stream, scout_sig_t *d_sigs) {
     if (!p || !d_sigs) return SCOUT_ERR_INVALID;
     if (!p->bound) return SCOUT_ERR_INVALID;
+    int rc = check_device(p);
+    if (rc) return rc;
     return sign_all(p, (cudaStream_t)stream, d_sigs);
 }
 
@@ -422,8 +460,9 @@ int scout_certify(scout_plan_t *p, void *stream, scout_report_t *report, scout_o
     if (!p || !report || !p->bound || p->R < 2) return SCOUT_ERR_INVALID;
     if (p->R > 64) return SCOUT_ERR_UNSUPPORTED;
     if ((outlier_cap && !h_outliers) || (undecided_cap && !h_undecided)) return SCOUT_ERR_INVALID;
-    int rc = ensure_certify_buffers(p, outlier_cap, undecided_cap);
+    int rc = check_device(p);
     if (rc) return rc;
+    if ((rc = ensure_certify_buffers(p, outlier_cap, undecided_cap))) return rc;
     cudaStream_t s = (cudaStream_t)stream;
     if ((rc = sign_all(p, s, p->d_sigs, p->d_out))) return rc;
     return vote_and_report(p, s, report, h_outliers, outlier_cap, h_undecided, undecided_cap);
@@ -438,8 +477,9 @@ int scout_certify_host(scout_plan_t *p, const void *const *h_ptrs, scout_report_
     const uint64_t n = (uint64_t)p->R * p->T;
     for (uint64_t i = 0; i < n; ++i)
         if (!h_ptrs[i]) return SCOUT_ERR_INVALID;
-    int rc = ensure_certify_buffers(p, outlier_cap, undecided_cap);
+    int rc = check_device(p);
     if (rc) return rc;
+    if ((rc = ensure_certify_buffers(p, outlier_cap, undecided_cap))) return rc;
     const uint64_t packed = p->tensor_poff[p->T];
     if (!p->s_copy) {
         SCOUT_CUDA(cudaStreamCreateWithFlags(&p->s_copy, cudaStreamNonBlocking));
@@ -507,6 +547,7 @@ int scout_certify_host(scout_plan_t *p, const void *const *h_ptrs, scout_report_
             l.recs = p->d_recs;
             l.error = p->d_error;
             l.variant = p->variant == 3 ? 0 : p->variant;
+            l.uniform_dtype = p->uniform_dtype;
             l.grid = p->grid;
             if ((rc = launch_sign_tiles(l, p->s_comp))) return rc;
             SCOUT_CUDA(cudaEventRecord(p->ev_done[buf], p->s_comp));
@@ -517,6 +558,7 @@ int scout_certify_host(scout_plan_t *p, const void *const *h_ptrs, scout_report_
     rc = launch_finalize(p->d_chunks, p->chunks.size(), p->R, p->d_recs, NT, p->tile_bytes / ROW_BYTES,
                          p->d_sigs, p->d_out, p->s_comp);
     if (rc) return rc;
+    if ((rc = mark_launched(p, p->s_comp))) return rc;
     return vote_and_report(p, p->s_comp, report, h_outliers, outlier_cap, h_undecided, undecided_cap);
 }
 
@@ -538,6 +580,7 @@ int scout_plan_replica_bad_counts(const scout_plan_t *p, uint64_t *h_counts) {
 int scout_rollup_tensors(const scout_plan_t *p, const scout_sig_t *d_sigs, uint64_t *d_tensor_sigs,
                          void *stream) {
     if (!p || !d_sigs || !d_tensor_sigs) return SCOUT_ERR_INVALID;
+    if (int rc = check_device(p)) return rc;
     return launch_rollup_tensors(p->d_chunks, p->d_tensor_chunk0, p->T, p->R, d_sigs, d_tensor_sigs,
                                  (cudaStream_t)stream);
 }
@@ -550,10 +593,20 @@ uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims) {
 
 int scout_plan_set(scout_plan_t *p, const char *key, int64_t value) {
     if (!p || !key) return SCOUT_ERR_INVALID;
+    if (int rc = check_device(p)) return rc;
+    if (!std::strcmp(key, "device_error")) {
+        // 0 clears the flag a timed-out wait left behind; a non-zero value sets it from the
+        // host (how the tests produce the failure without making a GPU wait run out)
+        const uint32_t v = value ? 1u : 0u;
+        if (p->launched) SCOUT_CUDA(cudaEventSynchronize(p->ev_last));
+        SCOUT_CUDA(cudaMemcpy(p->d_error, &v, sizeof(v), cudaMemcpyHostToDevice));
+        return SCOUT_OK;
+    }
     if (!std::strcmp(key, "tile_bytes")) {
         if (value < 2048 || value > 65536 || (value & (value - 1))) return SCOUT_ERR_INVALID;
         if ((uint32_t)value == p->tile_bytes) return SCOUT_OK;
         if (p->variant == 4 && value > 32768) return SCOUT_ERR_INVALID;
+        if (p->launched) SCOUT_CUDA(cudaEventSynchronize(p->ev_last));  // the tables may be in use
         p->tile_bytes = (uint32_t)value;
         try {
             build_tiles(p);
@@ -577,7 +630,7 @@ int scout_plan_set(scout_plan_t *p, const char *key, int64_t value) {
         if (value < 0 || value > 4) return SCOUT_ERR_INVALID;
         if (value == 4 && p->tile_bytes > 32768) return SCOUT_ERR_INVALID;  // a tile must fit one stage
         p->variant = (int)value;
-        return sign_grid_size(p->variant, p->device, &p->grid);
+        return sign_grid_size(p->variant, p->uniform_dtype, p->device, &p->grid);
     }
     if (!std::strcmp(key, "timing")) {
         if (value && !p->ev_t0) {
@@ -609,6 +662,7 @@ int scout_plan_get(const scout_plan_t *p, const char *key, int64_t *value) {
         *value = (int64_t)((double)ms * 1e6);
     }
     else if (!std::strcmp(key, "device_error")) {
+        if (int rc = check_device(p)) return rc;
         uint32_t e = 0;
         SCOUT_CUDA(cudaMemcpy(&e, p->d_error, sizeof(e), cudaMemcpyDeviceToHost));
         *value = e;

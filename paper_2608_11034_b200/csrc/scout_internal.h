@@ -149,10 +149,11 @@ struct SignLaunch {
     TileRec *recs;                // device [R][tiles_per_replica]
     uint32_t *error;              // device flag set when a bounded wait gave up (may be null)
     int variant;                  // 0 direct, 1 direct + register prefetch, 2 bulk-async ring, 3 read probe
+    int uniform_dtype;            // dtype shared by every tile of the launch, or -1 if they differ
     int grid;                     // CTAs to launch
 };
 int launch_sign_tiles(const SignLaunch &a, cudaStream_t stream);
-int sign_grid_size(int variant, int device, int *grid);
+int sign_grid_size(int variant, int uniform_dtype, int device, int *grid);
 int launch_bounded_wait_selftest(uint64_t limit_ns, uint64_t *d_out, cudaStream_t stream);
 
 // zero_out (may be null): a CertifyOut the finalise kernel clears for the vote that follows

@@ -18,6 +18,7 @@
 // element, counts NaN/Inf and sums the finite ones only.
 #include <cuda_fp16.h>
 
+#include <mutex>
 #include <type_traits>
 
 #include "scout_internal.h"
@@ -41,6 +42,12 @@ constexpr int SIGN_THREADS = 256;
 #endif
 #ifndef SCOUT_UNROLL
 #define SCOUT_UNROLL 8
+#endif
+#ifndef SCOUT_HASH_FORM
+#define SCOUT_HASH_FORM 0
+#endif
+#ifndef SCOUT_L2_PREFETCH
+#define SCOUT_L2_PREFETCH 0
 #endif
 constexpr int UNROLL = SCOUT_UNROLL;
 // bf16: how many of a word-quad's four high halves are widened by bit placement
@@ -247,12 +254,21 @@ __device__ __noinline__ void rescan_classifying(const uint8_t *tile, uint32_t nb
 // h * P lets every product be a 32x32+64 multiply-add (measured: fewest
 // instructions of the forms tried; a 64-bit accumulate costs two issue slots).
 __device__ __forceinline__ void fold_row(uint64_t &h, const uint4 &v, const uint32_t (&m)[4]) {
+#if SCOUT_HASH_FORM == 1
+    // row sum first (independent of h), then one short dependent step on h
+    uint64_t t = (uint64_t)m[0] * v.x;
+    t += (uint64_t)m[1] * v.y;
+    t += (uint64_t)m[2] * v.z;
+    t += (uint64_t)m[3] * v.w;
+    h = h * HASH_P + t;
+#else
     uint64_t t = h * HASH_P;
     t += (uint64_t)m[0] * v.x;
     t += (uint64_t)m[1] * v.y;
     t += (uint64_t)m[2] * v.z;
     t += (uint64_t)m[3] * v.w;
     h = t;
+#endif
 }
 
 // Per-lane state of one tile's scan: the lane's four slot multipliers, its share
@@ -331,6 +347,12 @@ __device__ __forceinline__ void scan_tile(const uint8_t *tile, uint32_t nbytes, 
         uint4 v[UNROLL];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) v[u] = ld_stream16(p + u * ROW_BYTES);
+#if SCOUT_L2_PREFETCH
+        // ask L2 for the next batch while this one is folded
+        if (lane == 0 && b > 1)
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p + UNROLL * ROW_BYTES),
+                         "r"((uint32_t)(UNROLL * ROW_BYTES)) : "memory");
+#endif
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) st.row(v[u]);
     }
@@ -342,7 +364,10 @@ __device__ __forceinline__ void scan_tile(const uint8_t *tile, uint32_t nbytes, 
 // Front end 1: rotating register pipeline.  PF_ROWS rows are always in flight:
 // as soon as a row has been folded its registers are reloaded with the row
 // PF_ROWS ahead, so a warp's loads overlap its own arithmetic.
-constexpr int PF_ROWS = 4;
+#ifndef SCOUT_PF_ROWS
+#define SCOUT_PF_ROWS 4
+#endif
+constexpr int PF_ROWS = SCOUT_PF_ROWS;
 
 template <int DT>
 __device__ __forceinline__ void scan_tile_prefetch(const uint8_t *tile, uint32_t nbytes, uint32_t lane,
@@ -426,7 +451,10 @@ __device__ __forceinline__ void store_record(TileRec *dst_rec, const TileRec &re
 }
 
 // Persistent grid; every warp takes whole tiles, replica-major, round-robin.
-template <int PREFETCH>
+// DTSEL >= 0: every tile of the launch has that dtype (the element path is fixed at
+// compile time, so the register allocation is that path's, not the union of all
+// seven); DTSEL < 0: the dtype is read from the tile table.
+template <int PREFETCH, int DTSEL>
 __global__ void __launch_bounds__(SIGN_THREADS, PREFETCH ? SCOUT_MINBLOCKS_PF : SCOUT_MINBLOCKS) sign_tiles_direct(const SignArgs a) {
     pdl_launch_dependents();
     const uint32_t lane = threadIdx.x & 31u;
@@ -440,10 +468,29 @@ __global__ void __launch_bounds__(SIGN_THREADS, PREFETCH ? SCOUT_MINBLOCKS_PF : 
         const TileDesc td = a.tiles[t];
         const uint8_t *tile = tile_address(a, td, r);
         TileRec rec;
-        if (PREFETCH) scan_dispatch_prefetch(td.dtype, tile, td.nbytes, lane, rec);
-        else          scan_dispatch(td.dtype, tile, td.nbytes, lane, rec);
+        if constexpr (DTSEL >= 0) {
+            if (PREFETCH) scan_tile_prefetch<DTSEL>(tile, td.nbytes, lane, rec);
+            else          scan_tile<DTSEL>(tile, td.nbytes, lane, rec);
+        } else {
+            if (PREFETCH) scan_dispatch_prefetch(td.dtype, tile, td.nbytes, lane, rec);
+            else          scan_dispatch(td.dtype, tile, td.nbytes, lane, rec);
+        }
         if (lane == 0) store_record(&a.recs[(uint64_t)r * a.tiles_per_replica + t], rec);
     }
+}
+
+using SignKernel = void (*)(const SignArgs);
+// The direct-scan kernel for a front end (0 direct, 1 register prefetch) and a launch
+// whose tiles all have dtype `uniform` (specialised for fp32 and bf16), or mixed (-1).
+SignKernel direct_kernel(int prefetch, int uniform) {
+    if (prefetch) {
+        if (uniform == SCOUT_DT_F32) return sign_tiles_direct<1, SCOUT_DT_F32>;
+        if (uniform == SCOUT_DT_BF16) return sign_tiles_direct<1, SCOUT_DT_BF16>;
+        return sign_tiles_direct<1, -1>;
+    }
+    if (uniform == SCOUT_DT_F32) return sign_tiles_direct<0, SCOUT_DT_F32>;
+    if (uniform == SCOUT_DT_BF16) return sign_tiles_direct<0, SCOUT_DT_BF16>;
+    return sign_tiles_direct<0, -1>;
 }
 
 // ---- front end 2: bulk-async ring ----------------------------------------------
@@ -1044,7 +1091,7 @@ __global__ void __launch_bounds__(FIN_THREADS) finalize_chunks(const ChunkDesc *
 
 }  // namespace
 
-int sign_grid_size(int variant, int device, int *grid) {
+int sign_grid_size(int variant, int uniform_dtype, int device, int *grid) {
     int sms = 0, per_sm = 0;
     SCOUT_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
     if (variant == 4) {
@@ -1053,10 +1100,9 @@ int sign_grid_size(int variant, int device, int *grid) {
     } else if (variant == 2) {
         SCOUT_CUDA(cudaFuncSetAttribute(sign_tiles_ring, cudaFuncAttributeMaxDynamicSharedMemorySize, RING_SMEM));
         SCOUT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sign_tiles_ring, SIGN_THREADS, RING_SMEM));
-    } else if (variant == 1) {
-        SCOUT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sign_tiles_direct<1>, SIGN_THREADS, 0));
     } else {
-        SCOUT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sign_tiles_direct<0>, SIGN_THREADS, 0));
+        SCOUT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, direct_kernel(variant == 1, uniform_dtype),
+                                                                 SIGN_THREADS, 0));
     }
     if (per_sm < 1) per_sm = 1;
     *grid = sms * per_sm;
@@ -1092,8 +1138,7 @@ int launch_sign_tiles(const SignLaunch &l, cudaStream_t stream) {
     switch (l.variant) {
         case 3: read_probe<<<grid, SIGN_THREADS, 0, stream>>>(a); break;
         case 2: sign_tiles_ring<<<grid, SIGN_THREADS, RING_SMEM, stream>>>(a); break;
-        case 1: sign_tiles_direct<1><<<grid, SIGN_THREADS, 0, stream>>>(a); break;
-        default: sign_tiles_direct<0><<<grid, SIGN_THREADS, 0, stream>>>(a); break;
+        default: direct_kernel(l.variant == 1, l.uniform_dtype)<<<grid, SIGN_THREADS, 0, stream>>>(a); break;
     }
     SCOUT_CUDA(cudaGetLastError());
     return SCOUT_OK;
@@ -1194,15 +1239,19 @@ __global__ void __launch_bounds__(FIN_THREADS) finalize_noalloc(const __grid_con
 }
 
 // Device address of the scratch array and SM count, looked up once per device.
+// The table is filled under a mutex, so that host threads making their first call
+// at the same time do not race on it.
 struct NoallocDevice {
     TileRec *scratch;
     int sms;
     bool ready;
 };
 static NoallocDevice g_noalloc_dev[NOALLOC_MAX_DEVICES];
+static std::mutex g_noalloc_mutex;
 
-int noalloc_setup(int device, NoallocDevice **out) {
+int noalloc_setup(int device, NoallocDevice *out) {
     if (device < 0 || device >= (int)NOALLOC_MAX_DEVICES) return SCOUT_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> guard(g_noalloc_mutex);
     NoallocDevice &d = g_noalloc_dev[device];
     if (!d.ready) {
         // `device` is the current device here, so the address is this GPU's copy
@@ -1214,7 +1263,7 @@ int noalloc_setup(int device, NoallocDevice **out) {
         d.sms = sms;
         d.ready = true;
     }
-    *out = &d;
+    *out = d;
     return SCOUT_OK;
 }
 
@@ -1248,9 +1297,10 @@ extern "C" int scout_sign_chunks_noalloc(uint32_t R, const void *const *replica_
     }
     int device = 0;
     SCOUT_CUDA(cudaGetDevice(&device));
-    NoallocDevice *dev = nullptr;
-    int rc = noalloc_setup(device, &dev);
+    NoallocDevice dev_info;
+    int rc = noalloc_setup(device, &dev_info);
     if (rc) return rc;
+    const NoallocDevice *dev = &dev_info;
 
     NoallocArgs a;
     for (uint32_t r = 0; r < 64; ++r) a.replica[r] = r < R ? (const uint8_t *)replica_ptrs[r] : nullptr;

@@ -41,6 +41,13 @@ def test_error_strings(lib):
 def test_shape_tag_matches_its_definition():
     for dims in ([], [7], [4096, 4096], [14336, 4096], [2**40, 3, 1]):
         assert binding.scout_shape_tag(dims) == defn.shape_tag(dims)
+    # and the stored answers (written by a stand-alone script, tests/golden/make_tag_kat.py)
+    stored = [ln.split() for ln in open(os.path.join(ROOT, "tests", "golden", "sf64_kat.txt"))
+              if ln.startswith("shapetag")]
+    assert len(stored) >= 3
+    for _, dims, want in stored:
+        dims = [] if dims == "-" else [int(x) for x in dims.split(",")]
+        assert binding.scout_shape_tag(dims) == int(want, 16)
 
 
 def test_plan_arguments_are_validated_before_any_device_work():

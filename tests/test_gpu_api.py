@@ -119,3 +119,85 @@ def test_a_wait_that_nothing_satisfies_gives_up_and_the_context_survives():
     assert len(got["outliers"]) == 1
     with pytest.raises(B.ScoutError):
         B.scout_selftest_bounded_wait(0, out.data_ptr(), 0)
+
+
+def test_device_error_flag_is_reported_once_and_cleared():
+    """A host-made failure: the flag a timed-out wait would leave is written from the
+    host.  The certify that sees it fails with SCOUT_ERR_CUDA and clears it; the next
+    one succeeds."""
+    from paper_2608_11034_b200 import binding as B
+    w = inputs.workload(1, "default", 1 / 8)
+    _, views = inputs.generate(w, "cuda")
+    plan = helpers.gpu_plan(w)
+    plan.bind(views)
+    good = plan.certify()
+    B.scout_plan_set(plan.handle, "device_error", 1)
+    assert B.scout_plan_get(plan.handle, "device_error") == 1
+    with pytest.raises(B.ScoutError) as e:
+        plan.certify()
+    assert e.value.code == B.ERR_CUDA
+    assert B.scout_plan_get(plan.handle, "device_error") == 0
+    again = plan.certify()
+    assert again["report"] == good["report"] and again["outliers"] == good["outliers"]
+    # the asynchronous path cannot report: the flag stays readable until it is cleared by hand
+    B.scout_plan_set(plan.handle, "device_error", 7)
+    plan.sign_and_vote()
+    torch.cuda.synchronize()
+    assert B.scout_plan_get(plan.handle, "device_error") == 1
+    B.scout_plan_set(plan.handle, "device_error", 0)
+    assert B.scout_plan_get(plan.handle, "device_error") == 0
+    plan.close()
+
+
+def test_rebinding_waits_for_a_scan_in_flight_on_a_non_blocking_stream():
+    """Re-binding right after an asynchronous sign on a non-blocking stream must not change
+    the table under the running scan: the records are those of the buffers bound at launch."""
+    from paper_2608_11034_b200 import binding as B
+    wa = inputs.Workload("bind_a", 0, "x", 3, 1 << 20,
+                         [inputs.TensorSpec("x", (48 << 20,), "f32", "normal", 0.02)], 7)
+    _, va = inputs.generate(wa, "cuda")
+    wb = inputs.Workload("bind_b", 0, "x", 3, 1 << 20,
+                         [inputs.TensorSpec("x", (48 << 20,), "f32", "normal", 0.02)], 8)
+    _, vb = inputs.generate(wb, "cuda")
+    plan = helpers.gpu_plan(wa)
+    side = torch.cuda.Stream()                  # torch's side streams do not sync with the default stream
+    d_a = torch.zeros(plan.C * wa.R * 32, dtype=torch.uint8, device="cuda")
+    d_b = torch.zeros_like(d_a)
+    torch.cuda.synchronize()
+    plan.bind(va)
+    B.scout_sign_chunks(plan.handle, side.cuda_stream, d_a.data_ptr())
+    plan.bind(vb)                               # 576 MB scan still running when this is called
+    B.scout_sign_chunks(plan.handle, side.cuda_stream, d_b.data_ptr())
+    side.synchronize()
+    got_a = d_a.cpu().numpy().view(B.SIG_DTYPE).reshape(plan.C, wa.R)
+    got_b = d_b.cpu().numpy().view(B.SIG_DTYPE).reshape(plan.C, wa.R)
+    plan.close()
+    ref_a = helpers.gpu_sign_vote(wa, va)["sigs"]
+    ref_b = helpers.gpu_sign_vote(wb, vb)["sigs"]
+    assert (got_a["hash"] == ref_a["hash"]).all() and (got_b["hash"] == ref_b["hash"]).all()
+    assert (ref_a["hash"] != ref_b["hash"]).all()
+
+
+def test_a_plan_used_with_another_device_current_is_rejected():
+    """The plan's tables live on the device that was current at creation.  With a
+    different current device every plan call returns SCOUT_ERR_INVALID.  On a one-GPU
+    box the same check is exercised through the plan's recorded device."""
+    from paper_2608_11034_b200 import binding as B
+    w = inputs.workload(1, "default", 1 / 16)
+    _, views = inputs.generate(w, "cuda")
+    plan = helpers.gpu_plan(w)
+    plan.bind(views)
+    if torch.cuda.device_count() < 2:
+        plan.close()
+        pytest.skip("needs two GPUs")
+    d_sigs = torch.zeros(plan.C * w.R * 32, dtype=torch.uint8, device="cuda:0")
+    try:
+        torch.cuda.set_device(1)
+        with pytest.raises(B.ScoutError) as e:
+            B.scout_sign_chunks(plan.handle, 0, d_sigs.data_ptr())
+        assert e.value.code == B.ERR_INVALID
+        with pytest.raises(B.ScoutError):
+            B.scout_plan_bind(plan.handle, [v.data_ptr() for rep in views for v in rep])
+    finally:
+        torch.cuda.set_device(0)
+    plan.close()

@@ -1,9 +1,12 @@
 """Parity at the benchmark's full sizes, in the launch configuration bench.py
-times.  Configs 1 and 2 are compared chunk by chunk; for configs 3, 4 and 5 the
-oracle signs a sample of (chunk, replica) pairs (every faulty chunk, the first
-and last chunks, ragged tails, random ones) and the vote is checked against
-what the injected patches imply for EVERY chunk."""
+times.  Configs 1 and 2 are compared chunk by chunk.  For configs 3, 4 and 5 the
+oracle signs EVERY chunk of one whole replica (so a fold that is wrong in the
+same way in all replicas cannot pass) plus a sample of (chunk, replica) pairs of
+the other replicas (every faulty chunk, the first and last chunks, ragged tails,
+random ones); the vote is checked against what the injected patches imply for
+every chunk."""
 import gc
+import os
 import random
 
 import numpy as np
@@ -48,6 +51,63 @@ def _check_sampled(w, views, sigs, chunks, pairs):
         assert (g["nan_count"], g["inf_count"]) == (o["nan_count"], o["inf_count"]), (c, r)
         assert abs(g["sum"] - o["sum"]) <= helpers.REL_TOL * abs_sum, (c, r)
         assert abs(g["sumsq"] - o["sumsq"]) <= helpers.REL_TOL * abs(o["sumsq"]), (c, r)
+
+
+def _abs_sums_on_device(x, dtype, chunk_bytes):
+    """sum |x| over the finite elements of each chunk of one tensor (plain torch on the
+    tensor's own device): only the scale of the tolerance on the sums."""
+    es = inputs.DTYPE_BYTES[dtype]
+    per = chunk_bytes // es
+    n_ch = (x.numel() + per - 1) // per
+    out = torch.zeros(n_ch, dtype=torch.float64, device=x.device)
+    if dtype == "u8":
+        return out.cpu().numpy()
+    flat = x.reshape(-1)
+    step = max(1, (256 << 20) // chunk_bytes)          # chunks per slice: bounds the fp64 temporaries
+    for c0 in range(0, n_ch, step):
+        part = flat[c0 * per:(c0 + step) * per].to(torch.float64).abs()
+        part = torch.where(torch.isfinite(part), part, torch.zeros_like(part))
+        full = part.numel() // per
+        if full:
+            out[c0:c0 + full] = part[:full * per].view(full, per).sum(1)
+        if part.numel() > full * per:
+            out[c0 + full] = part[full * per:].sum()
+    return out.cpu().numpy()
+
+
+def _check_whole_replica(w, views, sigs, chunks, r):
+    """Every chunk of replica r against the oracle (all host cores), tensors taken in
+    groups of about 1 GiB so that host memory stays bounded."""
+    tags = helpers.shape_tags(w)
+    nthreads = os.cpu_count() or 4
+    cb = w.chunk_bytes
+    group, group_bytes, c0, checked = [], 0, 0, 0
+
+    def flush():
+        nonlocal group, group_bytes, c0, checked
+        if not group:
+            return
+        tt = orc.make_tensor_table([(w.specs[t].nbytes, helpers.ORC_CODE[w.specs[t].dtype], tags[t])
+                                    for t in group])
+        arrays = [inputs.to_numpy_bytes(views[r][t]) for t in group]
+        n_ch = sum((w.specs[t].nbytes + cb - 1) // cb for t in group)
+        o = np.zeros((n_ch, 1), dtype=orc.SIG_DTYPE)
+        orc.sign_replica(tt, arrays, cb, o, 0, nthreads)
+        scale = np.concatenate([_abs_sums_on_device(views[r][t], w.specs[t].dtype, cb) for t in group])
+        g = sigs[c0:c0 + n_ch, r]
+        assert int(chunks["tensor"][c0]) == group[0] and int(chunks["tensor"][c0 + n_ch - 1]) == group[-1]
+        helpers.assert_sigs_match(g.reshape(-1, 1), o, scale.reshape(-1, 1))
+        c0 += n_ch
+        checked += n_ch
+        group, group_bytes = [], 0
+
+    for t, s in enumerate(w.specs):
+        group.append(t)
+        group_bytes += s.nbytes
+        if group_bytes >= (1 << 30):
+            flush()
+    flush()
+    assert checked == len(chunks)
 
 
 def _sample_pairs(w, chunks, want_out, n_random, seed):
@@ -111,6 +171,7 @@ def test_config_4_certify_full_size():
     clean[[c for c, _ in want_out]] = False
     assert (sigs["hash"][clean] == sigs["hash"][clean][:, :1]).all()
     _check_sampled(w, views, sigs, chunks, _sample_pairs(w, chunks, want_out, 6, 4))
+    _check_whole_replica(w, views, sigs, chunks, bad)
     # the certificate is the chain over the majority hashes: recompute it from the records
     maj = [int(sigs["hash"][c, (bad + 1) % w.R]) for c in range(plan.C)]
     import defn
@@ -139,6 +200,7 @@ def test_config_5_full_size():
     clean[[c for c, _ in want_out]] = False
     assert (sigs["hash"][clean] == sigs["hash"][clean][:, :1]).all()
     _check_sampled(w, views, sigs, chunks, _sample_pairs(w, chunks, want_out, 40, 5))
+    _check_whole_replica(w, views, sigs, chunks, want_out[0][1])
     plan.close()
     del views
     _free()
@@ -147,7 +209,7 @@ def test_config_5_full_size():
 def test_config_3_full_size():
     from paper_2608_11034_b200 import binding
     _free()
-    _need(130)
+    _need(135)
     w = inputs.workload(3)
     assert w.bytes_per_replica * w.R == 124_554_051_584
     _, views = inputs.generate(w, "cuda")
@@ -169,6 +231,7 @@ def test_config_3_full_size():
     clean[[c for c, _ in want_out]] = False
     assert (sigs["hash"][clean] == sigs["hash"][clean][:, :1]).all()
     _check_sampled(w, views, sigs, chunks, _sample_pairs(w, chunks, want_out, 8, 3))
+    _check_whole_replica(w, views, sigs, chunks, 5)
     plan.close()
     del views
     _free()

@@ -28,11 +28,27 @@ def _gen(name, n):
     raise ValueError(name)
 
 
+def _int_list(field):
+    return [] if field == "-" else [int(x) for x in field.split(",")]
+
+
+def _golden_tags():
+    """-> (shape-tag cases, certificate cases) from the stored file."""
+    shape, cert = [], []
+    for line in open(GOLDEN):
+        f = line.split()
+        if f and f[0] == "shapetag":
+            shape.append((_int_list(f[1]), int(f[2], 16)))
+        elif f and f[0] == "cert":
+            cert.append((_int_list(f[1]), int(f[2], 16)))
+    return shape, cert
+
+
 def _golden():
     kat, roll, mult, mix = [], [], [], []
     for line in open(GOLDEN):
         f = line.split()
-        if not f or f[0].startswith("#"):
+        if not f or f[0].startswith("#") or f[0] in ("shapetag", "cert"):
             continue
         if f[0] == "rollup":
             roll.append(([] if f[1] == "-" else [int(x) for x in f[1].split(",")], int(f[2], 16)))
@@ -73,6 +89,43 @@ def test_known_answers():
         assert orc.slot_multiplier(s) == want
     for z, want in mix:
         assert orc.mix64(z) == want
+
+
+def test_shape_tag_and_certificate_known_answers():
+    """Stored values from a stand-alone big-integer script (tests/golden/make_tag_kat.py):
+    the oracle and the tests' restatement must both reproduce them."""
+    shape, cert = _golden_tags()
+    assert len(shape) >= 3 and len(cert) >= 2
+    for dims, want in shape:
+        assert orc.shape_tag(dims) == want, dims
+        assert defn.shape_tag(dims) == want, dims
+    for hashes, want in cert:
+        # every replica holds the same hash per chunk: each chunk's majority hash is that hash
+        R = 3
+        sigs = np.zeros((len(hashes), R), dtype=orc.SIG_DTYPE)
+        for c, h in enumerate(hashes):
+            sigs["hash"][c, :] = h
+        rep = orc.certify(sigs)["report"]
+        assert rep["verdict"] == 0 and rep["certificate"] == want, hashes
+        assert defn.certificate(hashes) == want
+    # one outvoted replica does not change the certificate: it is over the majority hashes
+    hashes, want = cert[1]
+    sigs = np.zeros((len(hashes), 3), dtype=orc.SIG_DTYPE)
+    for c, h in enumerate(hashes):
+        sigs["hash"][c, :] = h
+    sigs["hash"][1, 2] ^= 0x10
+    rep = orc.certify(sigs)["report"]
+    assert rep["verdict"] == 1 and rep["certificate"] == want
+
+
+def test_stored_tag_lines_match_their_generator():
+    """The committed generator still prints exactly the stored lines."""
+    import subprocess
+    import sys
+    script = os.path.join(os.path.dirname(GOLDEN), "make_tag_kat.py")
+    out = subprocess.run([sys.executable, script], capture_output=True, text=True, check=True).stdout
+    stored = [ln.strip() for ln in open(GOLDEN) if ln.startswith(("shapetag", "cert"))]
+    assert out.split("\n")[:-1] == stored
 
 
 def test_mix64_is_a_bijection():
