@@ -1,38 +1,91 @@
-// Host-only part of the library: the checkpoint ledger of Sec. 8 (Algorithm 3)
-// and peer-group formation of Sec. 4.  No CUDA here.
+// Host-only part of the library: the checkpoint ledger of Sec. 8 (the protocol
+// Algorithm 3 summarises) and peer-group formation of Sec. 4.  No CUDA here.
 #include <new>
 
 #include "scout_ledger.h"
 
+// The ledger is two small machines (Sec. 8, "Checkpoint saving during training" and
+// "Checkpoint retrieval for failure recovery"):
+//   * a cycle of K accepted checks.  Closing a cycle shifts the durable roles by
+//     one place: what was persisted at the previous boundary has now seen a full
+//     catalog of accepted checks after its capture and becomes trusted; the newest
+//     capture is persisted in its place.
+//   * a selector that answers "which role do we restart from" for a failure class.
+//     It is a pure function of (failure class, machines reachable, emergency sweep
+//     result) and is kept as a decision table.
+struct DurableRoles {
+    uint64_t awaiting = SCOUT_NO_CHECKPOINT;  // persisted, not yet followed by a full accepted cycle
+    uint64_t trusted = SCOUT_NO_CHECKPOINT;   // persisted and followed by a full accepted cycle
+};
+
 struct scout_ledger {
-    uint64_t latest = SCOUT_NO_CHECKPOINT, candidate = SCOUT_NO_CHECKPOINT,
-             verified = SCOUT_NO_CHECKPOINT;
-    uint32_t q = 0, K = 1;
-    uint64_t n_persisted = 0;
+    uint64_t newest_capture = SCOUT_NO_CHECKPOINT;
+    DurableRoles durable;
+    uint32_t accepted_in_cycle = 0, cycle_length = 1;
+    uint64_t cycles_closed = 0;
 };
 
 namespace {
 
-// CheckpointRetrieval: which role answers failure class f.
-int choose(const scout_ledger *l, int f, int accessible, int sweep, scout_ledger_event_t *ev) {
-    ev->action = SCOUT_LEDGER_RETRIEVAL;
+enum class Verdict { Accept, Reject };  // does this boundary's outcome allow a capture?
+enum class Pick { Trusted, Newest, RunSweepFirst };
+
+// Only a numerical disagreement or a hang blocks the capture; slowness alone does not.
+Verdict judge(int outcome) {
+    return (outcome == SCOUT_OUTCOME_SDC || outcome == SCOUT_OUTCOME_HANG) ? Verdict::Reject
+                                                                         : Verdict::Accept;
+}
+
+// Decision table of the selector.  Rows: failure class.  Columns: machines
+// reachable? then the sweep result (not run / clean / found SDC).
+//   - a confirmed SDC never restarts from unverified state;
+//   - an unreachable machine hides part of the newest capture, so it cannot be vouched for;
+//   - a straggler is slow, not wrong: the newest capture is fine;
+//   - anything else is decided by replaying the whole catalog once.
+constexpr Pick T = Pick::Trusted, N = Pick::Newest, S = Pick::RunSweepFirst;
+constexpr Pick kSelector[5][2][3] = {
+    /* HEALTHY   */ {{T, T, T}, {S, N, T}},  // not a failure class; scout_ledger_retrieve rejects it
+    /* STRAGGLER */ {{T, T, T}, {N, N, N}},
+    /* SDC       */ {{T, T, T}, {T, T, T}},
+    /* HANG      */ {{T, T, T}, {S, N, T}},
+    /* OTHER     */ {{T, T, T}, {S, N, T}},
+};
+
+int select_restart_point(const scout_ledger *l, int failure, int reachable, int sweep,
+                         scout_ledger_event_t *ev) {
+    const int sweep_col = sweep < 0 ? 0 : (sweep == 0 ? 1 : 2);
+    const Pick pick = kSelector[failure][reachable ? 1 : 0][sweep_col];
     ev->promoted = SCOUT_NO_CHECKPOINT;
-    bool use_verified;
-    if (f == SCOUT_OUTCOME_SDC || !accessible) {
-        use_verified = true;
-    } else if (f == SCOUT_OUTCOME_STRAGGLER) {
-        use_verified = false;
-    } else if (sweep < 0) {  // the full-catalog replay has to run before a choice is possible
-        ev->action = SCOUT_LEDGER_NEED_SWEEP;
-        ev->role = SCOUT_ROLE_NONE;
-        ev->checkpoint = SCOUT_NO_CHECKPOINT;
-        return SCOUT_OK;
-    } else {
-        use_verified = sweep != 0;
+    switch (pick) {
+        case Pick::RunSweepFirst:
+            ev->action = SCOUT_LEDGER_NEED_SWEEP;
+            ev->role = SCOUT_ROLE_NONE;
+            ev->checkpoint = SCOUT_NO_CHECKPOINT;
+            break;
+        case Pick::Trusted:
+            ev->action = SCOUT_LEDGER_RETRIEVAL;
+            ev->role = SCOUT_ROLE_VERIFIED;
+            ev->checkpoint = l->durable.trusted;
+            break;
+        case Pick::Newest:
+            ev->action = SCOUT_LEDGER_RETRIEVAL;
+            ev->role = SCOUT_ROLE_LATEST;
+            ev->checkpoint = l->newest_capture;
+            break;
     }
-    ev->role = use_verified ? SCOUT_ROLE_VERIFIED : SCOUT_ROLE_LATEST;
-    ev->checkpoint = use_verified ? l->verified : l->latest;
     return SCOUT_OK;
+}
+
+// The K-th accepted check of a cycle arrived: shift the durable roles.
+void close_cycle(scout_ledger *l, scout_ledger_event_t *ev) {
+    const DurableRoles before = l->durable;
+    l->durable.trusted = before.awaiting;
+    l->durable.awaiting = l->newest_capture;  // the caller persists this id
+    l->accepted_in_cycle = 0;
+    l->cycles_closed += 1;
+    ev->action = SCOUT_LEDGER_BOUNDARY;
+    ev->checkpoint = l->durable.awaiting;
+    ev->promoted = l->durable.trusted;
 }
 
 bool valid_outcome(int f) { return f >= SCOUT_OUTCOME_HEALTHY && f <= SCOUT_OUTCOME_OTHER; }
@@ -67,7 +120,7 @@ int scout_ledger_create(uint32_t K, scout_ledger_t **out) {
     if (K == 0) return SCOUT_ERR_INVALID;
     scout_ledger *l = new (std::nothrow) scout_ledger;
     if (!l) return SCOUT_ERR_NOMEM;
-    l->K = K;
+    l->cycle_length = K;
     *out = l;
     return SCOUT_OK;
 }
@@ -79,42 +132,34 @@ int scout_ledger_destroy(scout_ledger_t *l) {
 
 int scout_ledger_state(const scout_ledger_t *l, scout_ledger_state_t *s) {
     if (!l || !s) return SCOUT_ERR_INVALID;
-    s->latest = l->latest;
-    s->candidate = l->candidate;
-    s->verified = l->verified;
-    s->q = l->q;
-    s->K = l->K;
-    s->n_persisted = l->n_persisted;
+    s->latest = l->newest_capture;
+    s->candidate = l->durable.awaiting;
+    s->verified = l->durable.trusted;
+    s->q = l->accepted_in_cycle;
+    s->K = l->cycle_length;
+    s->n_persisted = l->cycles_closed;
     return SCOUT_OK;
 }
 
 int scout_ledger_save(scout_ledger_t *l, int f, uint64_t captured, int accessible, int sweep,
                       scout_ledger_event_t *ev) {
     if (!l || !ev || !valid_outcome(f)) return SCOUT_ERR_INVALID;
-    if (f == SCOUT_OUTCOME_SDC || f == SCOUT_OUTCOME_HANG) return choose(l, f, accessible, sweep, ev);
+    if (judge(f) == Verdict::Reject)  // nothing is captured; the ledger itself is left as it is
+        return select_restart_point(l, f, accessible, sweep, ev);
     if (captured == SCOUT_NO_CHECKPOINT) return SCOUT_ERR_INVALID;
-    l->latest = captured;
-    l->q += 1;
+    l->newest_capture = captured;
     ev->action = SCOUT_LEDGER_CAPTURED;
     ev->role = SCOUT_ROLE_NONE;
     ev->checkpoint = SCOUT_NO_CHECKPOINT;
     ev->promoted = SCOUT_NO_CHECKPOINT;
-    if (l->q == l->K) {
-        l->q = 0;
-        l->verified = l->candidate;
-        l->candidate = l->latest;  // persisted by the caller
-        l->n_persisted += 1;
-        ev->action = SCOUT_LEDGER_BOUNDARY;
-        ev->checkpoint = l->candidate;
-        ev->promoted = l->verified;
-    }
+    if (++l->accepted_in_cycle == l->cycle_length) close_cycle(l, ev);
     return SCOUT_OK;
 }
 
 int scout_ledger_retrieve(const scout_ledger_t *l, int f, int accessible, int sweep,
                           scout_ledger_event_t *ev) {
     if (!l || !ev || !valid_outcome(f) || f == SCOUT_OUTCOME_HEALTHY) return SCOUT_ERR_INVALID;
-    return choose(l, f, accessible, sweep, ev);
+    return select_restart_point(l, f, accessible, sweep, ev);
 }
 
 int scout_outcome_from_report(const scout_report_t *r, int *outcome) {

@@ -28,6 +28,32 @@ def test_oracle_two_recipe_trace_of_the_paper():
     assert (L.latest, L.candidate, L.verified) == (4, 4, 2)        # nothing captured at step 5
 
 
+def test_oracle_hand_derived_traces_k1_and_k3():
+    """Worked by hand from the prose of Sec. 8.  K = 1 (static shapes): every accepted
+    check closes a cycle, so the capture one boundary back is the verified one.  K = 3:
+    captures 3 and 6 are persisted; 3 is verified once check 6 has been accepted."""
+    L = H.Ledger(1)
+    assert L.checkpoint_save(H.HEALTHY, 10) == ("boundary", 10, None)
+    assert L.checkpoint_save(H.STRAGGLER, 11) == ("boundary", 11, 10)       # a completed straggler counts
+    assert L.checkpoint_save(H.HANG, 12, True, None) == ("retrieval", "need_sweep", None)
+    assert L.checkpoint_save(H.HANG, 12, True, False) == ("retrieval", "latest", 11)
+    assert (L.latest, L.candidate, L.verified, L.q) == (11, 11, 10, 0)
+    assert L.checkpoint_save(H.HEALTHY, 13) == ("boundary", 13, 11)
+
+    L = H.Ledger(3)
+    want = {1: ("captured",), 2: ("captured",), 3: ("boundary", 3, None), 4: ("captured",),
+            5: ("captured",), 6: ("boundary", 6, 3), 7: ("captured",)}
+    for step in range(1, 8):
+        assert L.checkpoint_save(H.HEALTHY, step) == want[step]
+    assert (L.latest, L.candidate, L.verified, L.q) == (7, 6, 3, 1)
+    assert L.checkpoint_save(H.SDC, 8) == ("retrieval", "verified", 3)      # not 6: only one cycle followed it
+    assert (L.latest, L.candidate, L.verified, L.q) == (7, 6, 3, 1)         # and nothing moved
+    assert L.checkpoint_retrieval(H.STRAGGLER) == ("latest", 7)
+    # an SDC in the middle of a cycle does not restart the count (the listing leaves q alone)
+    assert L.checkpoint_save(H.HEALTHY, 9) == ("captured",)
+    assert L.checkpoint_save(H.HEALTHY, 10) == ("boundary", 10, 6)
+
+
 def test_oracle_retrieval_rules_from_the_prose():
     L = H.Ledger(1)
     for step in (1, 2, 3):
