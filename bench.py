@@ -41,6 +41,7 @@ FALLBACK_HBM_GBS = 6650.0
 # 1.8000 GB scanned (fp32), 1.1407 + 0.016 for 1.1401 GB (bf16).  Traffic grows
 # in proportion to the bytes scanned, so a full-size launch is scaled by this.
 SCAN_TRAFFIC_RATIO = 1.0148
+SCAN_TRAFFIC_SOURCE = "ncu capture of the scan kernel on 1.8 GB, scaled to the launch (profiles/)"
 
 
 def measured_peak():
@@ -65,6 +66,9 @@ def parse_args():
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--variant", type=int, default=None)
     ap.add_argument("--tile-bytes", type=int, default=None)
+    ap.add_argument("--also", default=None,
+                    help="comma-separated configs measured after the headline one and reported under "
+                         "'also' (default: 3,5 for the default full-size run at N=1; '' for none)")
     return ap.parse_args()
 
 
@@ -183,8 +187,10 @@ def run_reference(args):
     orc.build()
     w = inputs.workload(args.config, BENCH_CASE.get(args.config, "default"), args.scale)
     cores = os.cpu_count() or 1
-    # generate only what is sampled: shrink each tensor to its leading chunks
-    budget = 192 << 20
+    # generate only what is sampled: shrink each tensor to its leading chunks.  The sample
+    # holds at least four chunks per host thread, so that every thread has work (a smaller
+    # sample under-reports the oracle), and at most 2 GiB per step.
+    budget = min(max(192 << 20, 4 * cores * w.chunk_bytes), 2 << 30)
     per_tensor = max(w.chunk_bytes, budget // len(w.specs) // w.chunk_bytes * w.chunk_bytes)
     specs, total = [], 0
     for s in w.specs:
@@ -210,10 +216,13 @@ def run_reference(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / len(times),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64+f64",
         "data": "synthetic",
-        "config": {"workload": w.name, "R": w.R, "chunk_bytes": w.chunk_bytes,
-                   "sample_bytes_per_step": total},
+        "config": dict(config_block(w, sum((x.nbytes + w.chunk_bytes - 1) // w.chunk_bytes for x in w.specs)),
+                       parallelism="single GPU" if args.gpus == 1 else f"{args.gpus} independent replica sets"),
+        "sample_bytes_per_step": total,
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
-                         "sample": f"one replica's leading chunks, {total} bytes per step, {cores} threads"},
+                         "sample": f"one replica's leading chunks, {total} bytes per step, {cores} threads; "
+                                   f"the CUDA arm's cpu_baseline leg times the same oracle once over a "
+                                   f"larger sample of the resident data"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -239,25 +248,20 @@ def expected_pairs(w, plan_handle, binding, inputs):
     return sorted(pairs)
 
 
-def main():
-    args = parse_args()
-    if args.impl == "reference":
-        return run_reference(args)
+def config_block(w, C):
+    """Names the workload; the same keys in both arms (no launch settings here)."""
+    return {"workload": w.name, "R": w.R, "tensors": len(w.specs), "chunks": C,
+            "chunk_bytes": w.chunk_bytes, "bytes_per_step_per_gpu": w.R * w.bytes_per_replica}
 
-    import numpy as np
+
+def run_config(cfg, args, rank, world, local, headline):
+    """One config on this rank's GPU: warm-up, K timed steps (CUDA events on the current
+    stream, max over ranks), the scan kernel's own time for every one of those steps,
+    the read-only probe, and the check of the last step's answer.  -> dict."""
     import torch
-    import torch.distributed as dist
     from paper_2608_11034_b200 import binding, dist_util, inputs
 
-    rank, world, local = dist_util.rank_info()
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (the product path has no CPU fallback)")
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist_util.init("nccl", torch.device("cuda", local))
-    barrier = dist_util.barrier
-
-    w = inputs.workload(args.config, BENCH_CASE.get(args.config, "default"), args.scale)
+    w = inputs.workload(cfg, BENCH_CASE.get(cfg, "default"), args.scale)
     w.seed = dist_util.rank_seed(w.seed, rank)   # every rank scans its own replica set
     flats, views = inputs.generate(w, "cuda")
     total_bytes = w.R * w.bytes_per_replica
@@ -269,10 +273,8 @@ def main():
         binding.scout_plan_set(plan.handle, "tile_bytes", args.tile_bytes)
     if args.variant is not None:
         binding.scout_plan_set(plan.handle, "variant", args.variant)
-    binding.scout_plan_set(plan.handle, "timing", 1)
     plan.bind(views)
-    use_certify = args.config == 4
-    stream = torch.cuda.current_stream().cuda_stream
+    use_certify = cfg == 4
 
     def step():
         if use_certify:
@@ -283,12 +285,12 @@ def main():
     for _ in range(max(args.warmup, 0)):
         step()
     torch.cuda.synchronize()
+    binding.scout_plan_set(plan.handle, "timing", 1)      # from here on every scan launch is timed
 
     sampler = ClockSampler(local) if rank == 0 else None
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
           for _ in range(args.steps)]
-    scan_ns = []
-    barrier()
+    dist_util.barrier()
     torch.cuda.synchronize()
     for i in range(args.steps):
         if flush is not None:
@@ -296,41 +298,40 @@ def main():
         ev[i][0].record()
         last = step()
         ev[i][1].record()
-        if use_certify or small:
-            torch.cuda.synchronize()
-            scan_ns.append(binding.scout_plan_get(plan.handle, "last_sign_ns"))
     torch.cuda.synchronize()
-    barrier()
+    dist_util.barrier()
     clocks = sampler.stop() if sampler else None
-    if not scan_ns:
-        scan_ns.append(binding.scout_plan_get(plan.handle, "last_sign_ns"))
-    ms = dist_util.max_over_ranks(sum(a.elapsed_time(b) for a, b in ev), "cuda")
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    ms = dist_util.max_over_ranks(sum(step_ms), "cuda")
+    n_scan = binding.scout_plan_get(plan.handle, "timed_sign_launches")
+    scan_ns = binding.scout_plan_get(plan.handle, "timed_sign_ns")
+    # the ring holds the last 256 launches: with more steps than that, compare like with like
+    steps_cmp = step_ms[-n_scan:]
+    if n_scan != min(args.steps, 256) or scan_ns * 1e-6 > sum(steps_cmp) * 1.0005:
+        raise SystemExit(f"inconsistent timing: {n_scan} scan launches took {scan_ns * 1e-6:.3f} ms inside "
+                         f"steps that took {sum(steps_cmp):.3f} ms")
 
     # the last timed step must have produced the right answer
     want = expected_pairs(w, plan.handle, binding, inputs)
     if use_certify:
-        got = last["outliers"]
-        verdict = last["report"]["verdict"]
+        got, verdict = last["outliers"], last["report"]["verdict"]
     else:
-        res = plan.fetch()
-        got = res["outliers"]
-        verdict = None
-    verified = got == want
-    if not verified:
-        raise SystemExit(f"wrong result: outliers {got[:8]} expected {want[:8]}")
+        got, verdict = plan.fetch()["outliers"], None
+    if got != want:
+        raise SystemExit(f"{w.name}: wrong result: outliers {got[:8]} expected {want[:8]}")
 
-    value = dist_util.aggregate_gbs(total_bytes, world, args.steps, ms)
     peak, peak_kind = measured_peak()
-    scan_s = (sum(scan_ns) / len(scan_ns)) * 1e-9
+    scan_s = scan_ns * 1e-9 / n_scan
     achieved = total_bytes / scan_s / 1e9
-    C = plan.C
     roofline = {
         "bound": "hbm", "kernel": "sign_tiles", "achieved": achieved, "peak": peak, "unit": "GB/s",
         "frac": achieved / peak, "peak_kind": peak_kind,
         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
         "algorithmic_bytes_per_launch": total_bytes,
-        "avg_launch_ms": scan_s * 1e3, "launches_timed": len(scan_ns),
+        "avg_launch_ms": scan_s * 1e3, "launches_timed": n_scan,
+        "scan_share_of_step_time": scan_ns * 1e-6 / sum(steps_cmp),
         "traffic": (SCAN_TRAFFIC_RATIO * total_bytes) if SCAN_TRAFFIC_RATIO else None,
+        "traffic_source": SCAN_TRAFFIC_SOURCE,
     }
 
     # read-only probe on the same plan and buffers: what the memory system delivers to
@@ -362,64 +363,64 @@ def main():
         msw = sum(a0.elapsed_time(a1) for a0, a1 in evw)
         warm = {"value": total_bytes * args.steps / (msw * 1e-3) / 1e9, "ms_per_step": msw / args.steps}
 
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "u64+f64", "data": "synthetic",
-        "config": {"workload": w.name, "R": w.R, "tensors": len(w.specs), "chunks": C,
-                   "chunk_bytes": w.chunk_bytes, "bytes_per_step_per_gpu": total_bytes,
-                   "call": "scout_certify" if use_certify else "scout_sign_chunks+scout_consensus_vote",
+    value = dist_util.aggregate_gbs(total_bytes, world, args.steps, ms)
+    out = {
+        "value": value, "ms_per_step": ms / args.steps,
+        "config": config_block(w, plan.C),
+        "launch": {"call": "scout_certify" if use_certify else "scout_sign_chunks+scout_consensus_vote",
+                   "kernels_per_step": binding.scout_plan_get(plan.handle, "certify_kernels") if use_certify
+                   else binding.scout_plan_get(plan.handle, "sign_kernels") + 1,
                    "tile_bytes": binding.scout_plan_get(plan.handle, "tile_bytes"),
                    "variant": binding.scout_plan_get(plan.handle, "variant"),
                    "l2": "512 MiB written between steps" if small else "inputs far larger than L2, no flush",
-                   "parallelism": f"{world} independent replica sets" if world > 1 else "single GPU"},
+                   "timed_region_s": ms * 1e-3,
+                   "regime": "burst clocks (timed region under 1 s)" if ms < 1000 else "sustained"},
         "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
         "frac_of_measured_copy": value / world / peak,
-        "verified": verified, "verdict": verdict,
-        "gpu_launches": 4 * args.steps if use_certify else 3 * args.steps,
-        "clocks": clocks, "roofline": roofline, "l2_warm": warm,
+        "verified": True, "verdict": verdict, "clocks": clocks, "roofline": roofline, "l2_warm": warm,
     }
 
     # ---- end to end: replicas in pinned host memory, copies inside the timed region
-    if not args.no_e2e and rank == 0 and world == 1:
-        try:
-            bad = sorted({p.replica for p in w.patches})
-            base = torch.empty(flats[0].numel(), dtype=torch.uint8, pin_memory=True)
-            clean = next(r for r in range(w.R) if r not in bad)
-            base.copy_(flats[clean])
-            host = {r: base for r in range(w.R) if r not in bad}
-            for r in bad:
-                h = torch.empty(flats[0].numel(), dtype=torch.uint8, pin_memory=True)
-                h.copy_(flats[r])
-                host[r] = h
-            hviews = [inputs.tensor_views(host[r], w.specs) for r in range(w.R)]
-            hptrs = [v.data_ptr() for rep in hviews for v in rep]
-            binding.scout_certify_host(plan.handle, hptrs)          # warm-up (allocates staging)
-            t0 = time.perf_counter()
-            for _ in range(args.e2e_steps):
-                rep = binding.scout_certify_host(plan.handle, hptrs)
-            dt = time.perf_counter() - t0
-            assert rep["outliers"] == want
-            line["e2e"] = {"value": total_bytes * args.e2e_steps / dt / 1e9, "unit": UNIT,
-                           "h2d_bytes_per_step": total_bytes,
-                           "d2h_bytes_per_step": 576 + 16 * len(want),
-                           "steps": args.e2e_steps, "call": "scout_certify_host",
-                           "host_memory": f"pinned; {len(bad) + 1} distinct replica images "
-                                          f"(clean replicas share one host image)"}
-            del base, host, hviews
-        except Exception as e:                                       # noqa: BLE001
-            line["e2e"] = {"value": None, "unit": UNIT, "error": repr(e)[:200]}
-    else:
-        line["e2e"] = {"value": None, "unit": UNIT, "note": "measured on rank 0 at N=1 only"}
+    if headline:
+        if not args.no_e2e and rank == 0 and world == 1:
+            try:
+                bad = sorted({p.replica for p in w.patches})
+                base = torch.empty(flats[0].numel(), dtype=torch.uint8, pin_memory=True)
+                clean = next(r for r in range(w.R) if r not in bad)
+                base.copy_(flats[clean])
+                host = {r: base for r in range(w.R) if r not in bad}
+                for r in bad:
+                    h = torch.empty(flats[0].numel(), dtype=torch.uint8, pin_memory=True)
+                    h.copy_(flats[r])
+                    host[r] = h
+                hviews = [inputs.tensor_views(host[r], w.specs) for r in range(w.R)]
+                hptrs = [v.data_ptr() for rep in hviews for v in rep]
+                binding.scout_certify_host(plan.handle, hptrs)          # warm-up (allocates staging)
+                t0 = time.perf_counter()
+                for _ in range(args.e2e_steps):
+                    rep = binding.scout_certify_host(plan.handle, hptrs)
+                dt = time.perf_counter() - t0
+                assert rep["outliers"] == want
+                out["e2e"] = {"value": total_bytes * args.e2e_steps / dt / 1e9, "unit": UNIT,
+                              "h2d_bytes_per_step": total_bytes,
+                              "d2h_bytes_per_step": 576 + 16 * len(want),
+                              "steps": args.e2e_steps, "call": "scout_certify_host",
+                              "host_memory": f"pinned; {len(bad) + 1} distinct replica images "
+                                             f"(clean replicas share one host image)"}
+                del base, host, hviews
+            except Exception as e:                                       # noqa: BLE001
+                out["e2e"] = {"value": None, "unit": UNIT, "error": repr(e)[:200]}
+        else:
+            out["e2e"] = {"value": None, "unit": UNIT, "note": "measured on rank 0 at N=1 only"}
 
     # ---- CPU oracle on a bounded sample, with a parity spot check against the CUDA records
     if not args.no_cpu_baseline and rank == 0 and world == 1:
         from oracle import scout_oracle as orc
         orc.build()
-        cb, (tt, picked, osigs) = cpu_baseline(w, views, args.cpu_seconds)
+        cb, (tt, picked, osigs) = cpu_baseline(w, views, args.cpu_seconds if headline else args.cpu_seconds / 3)
         plan.sign()                              # records into a torch-owned buffer
         torch.cuda.synchronize()
-        all_sigs = plan.d_sigs.cpu().numpy().view(binding.SIG_DTYPE).reshape(C, w.R)
+        all_sigs = plan.d_sigs.cpu().numpy().view(binding.SIG_DTYPE).reshape(plan.C, w.R)
         first, c = {}, 0
         for t, s in enumerate(w.specs):
             first[t] = c
@@ -433,13 +434,115 @@ def main():
                 ok &= abs(g["sumsq"] - o["sumsq"]) <= 1e-12 * abs(o["sumsq"])
                 oc += 1
         cb["parity_spot_check"] = {"chunks": oc, "ok": bool(ok)}
-        line["cpu_baseline"] = cb
+        out["cpu_baseline"] = cb
         if not ok:
-            raise SystemExit("CUDA records disagree with the oracle on the sampled chunks")
+            raise SystemExit(f"{w.name}: CUDA records disagree with the oracle on the sampled chunks")
     else:
-        line["cpu_baseline"] = None
+        out["cpu_baseline"] = None
 
     plan.close()
+    del plan, views, flats, flush
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+    return out
+
+
+def run_distributed(args, rank, world, local):
+    """The deployed form of C3 on config 4's state: ONE replica per GPU (R = N), each
+    rank signs its own 12 GB, the [C] records are all-gathered over NCCL, every rank
+    votes on the gathered table.  Same metric: bytes all ranks scanned / slowest rank."""
+    import torch
+    from paper_2608_11034_b200 import binding, dist_c3, dist_util, inputs
+
+    w = inputs.workload(4, "default", args.scale)       # same seed on every rank: equivalent replicas
+    flat, views = inputs.generate_replica0(w, "cuda")
+    mine = [inputs.Patch(0, p.tensor, p.element, p.op, p.value) for p in w.patches if p.replica % world == rank]
+    inputs.apply_patches([views], w.specs, mine)
+    c3 = dist_c3.DistributedC3(binding.make_tensor_table(w.specs), w.chunk_bytes)
+    c3.bind(views)
+    for _ in range(max(args.warmup, 0)):
+        c3.step()
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    dist_util.barrier()
+    torch.cuda.synchronize()
+    for a, b in ev:
+        a.record(); c3.step(); b.record()
+    torch.cuda.synchronize()
+    dist_util.barrier()
+    ms = dist_util.max_over_ranks(sum(a.elapsed_time(b) for a, b in ev), "cuda")
+    got = c3.fetch()
+    # chunks that hold a patch must be the ones named (attributed with R >= 3; with R = 2 a
+    # difference cannot be attributed and the chunk is listed as undecided)
+    per_tensor = (w.specs[0].nbytes + w.chunk_bytes - 1) // w.chunk_bytes
+    want = sorted({p.tensor * per_tensor + (p.element * 4) // w.chunk_bytes for p in w.patches})
+    named = sorted({c for c, _ in got["outliers"]} | set(got["undecided"]))
+    if named != want:
+        raise SystemExit(f"distributed C3: chunks named {named}, expected {want}")
+    c3.close()
+    return {"value": world * w.bytes_per_replica * args.steps / (ms * 1e-3) / 1e9, "unit": UNIT,
+            "ms_per_step": ms / args.steps, "R": world, "bytes_per_rank_per_step": w.bytes_per_replica,
+            "gathered_bytes_per_rank": c3.C * 32, "transport": "nccl all_gather_into_tensor",
+            "chunks_named": named, "form": "one replica per GPU: sign, all-gather records, vote on every rank"}
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2608_11034_b200 import dist_util
+
+    rank, world, local = dist_util.rank_info()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the product path has no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist_util.init("nccl", torch.device("cuda", local))
+
+    head = run_config(args.config, args, rank, world, local, headline=True)
+    line = {
+        "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": head["ms_per_step"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u64+f64", "data": "synthetic",
+        "config": dict(head["config"], parallelism=f"{world} independent replica sets" if world > 1 else "single GPU"),
+        "launch": head["launch"],
+        "frac_of_nominal_8TBs": head["frac_of_nominal_8TBs"],
+        "frac_of_measured_copy": head["frac_of_measured_copy"],
+        "verified": head["verified"], "verdict": head["verdict"],
+        "gpu_launches": head["launch"]["kernels_per_step"] * args.steps,
+        "clocks": head["clocks"], "roofline": head["roofline"], "l2_warm": head["l2_warm"],
+        "e2e": head["e2e"], "cpu_baseline": head["cpu_baseline"],
+    }
+
+    # The other two large configs (bf16 parameters; 10,000 mixed tensors), measured the same
+    # way after the headline config's buffers have been freed.
+    if args.also is None:
+        also = [3, 5] if (args.config == 4 and args.scale == 1.0 and world == 1) else []
+    else:
+        also = [int(x) for x in args.also.split(",") if x]
+    if also:
+        line["also"] = {}
+        for cfg in also:
+            r = run_config(cfg, args, rank, world, local, headline=False)
+            line["also"][r["config"]["workload"]] = {
+                "value": r["value"], "ms_per_step": r["ms_per_step"],
+                "bytes_per_step": r["config"]["bytes_per_step_per_gpu"],
+                "frac_of_nominal_8TBs": r["frac_of_nominal_8TBs"],
+                "roofline": {k: r["roofline"][k] for k in ("achieved", "frac", "avg_launch_ms", "launches_timed",
+                                                          "scan_share_of_step_time", "read_probe_gbs",
+                                                          "frac_of_read_probe")},
+                "clocks": r["clocks"], "verified": r["verified"], "regime": r["launch"]["regime"],
+                "parity_spot_check": (r["cpu_baseline"] or {}).get("parity_spot_check"),
+                "cpu_oracle_gbs": (r["cpu_baseline"] or {}).get("value"),
+            }
+
+    if world > 1:       # the paper's deployment form, next to the independent-sets number above
+        line["distributed_c3"] = run_distributed(args, rank, world, local)
+
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:

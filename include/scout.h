@@ -260,10 +260,14 @@ SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/)
  *                     3 = read-only probe (measures the memory system only: the
  *                     records it leaves are NOT signatures)
  *   set "grid"        CTAs of the scan kernel
- *   set "timing"      1: record CUDA events around the scan kernel on the
- *                     caller's stream
+ *   set "timing"      1: record a pair of CUDA events around every scan kernel on
+ *                     the caller's stream (a ring of 256 pairs); setting it again
+ *                     restarts the count
  *   get "last_sign_ns" device time of the most recent scan kernel (needs
  *                     "timing" and a synchronised stream)
+ *   get "timed_sign_launches", "timed_sign_ns"  number of scan launches since
+ *                     "timing" was set that the ring still holds (at most 256) and
+ *                     their total device time (synchronised stream)
  *   get "device_error" 1 if a kernel's bounded wait gave up since the flag was last
  *                     cleared (synchronises); the records of such a run are not
  *                     valid.  scout_certify and scout_certify_host report it as
@@ -271,6 +275,8 @@ SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/)
  *                     (asynchronous, so it cannot report) read it here.
  *   set "device_error" 0 clears the flag; a non-zero value sets it from the host
  *                     (a way to exercise the error path without a GPU fault)
+ *   get "sign_kernels", "certify_kernels"  kernels one scout_sign_chunks / one
+ *                     scout_certify call launches for this plan
  *   get "n_tiles", "scratch_bytes", and every settable key
  * Results do not depend on tile_bytes, variant or grid except for the rounding
  * order of the floating-point sums. */

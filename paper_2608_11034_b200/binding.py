@@ -23,6 +23,7 @@ OK, ERR_INVALID, ERR_ALIGN, ERR_UNSUPPORTED, ERR_CUDA, ERR_NOMEM, ERR_TRUNCATED 
 DT_U8, DT_F32, DT_BF16, DT_I64, DT_F16, DT_F64, DT_I32 = range(7)
 AGREE, ATTRIBUTED, INCONCLUSIVE = 0, 1, 2
 CERTIFIED, VERDICT_ATTRIBUTED, UNDECIDED = 0, 1, 2
+MAX_REPLICAS = 1024          # SCOUT_MAX_REPLICAS of scout.h
 DTYPE_CODE = {"u8": DT_U8, "f32": DT_F32, "bf16": DT_BF16, "i64": DT_I64, "f16": DT_F16,
               "f64": DT_F64, "i32": DT_I32}
 

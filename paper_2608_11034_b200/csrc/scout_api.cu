@@ -36,6 +36,7 @@ using namespace scout;
 
 // Pinned landing area of scout_certify's device-to-host copies.
 constexpr uint64_t CERTIFY_HEAD = 64;
+constexpr size_t TIMING_RING = 256;  // event pairs kept for the "timing" knob
 struct CertifyHost {
     CertifyOut out;
     uint32_t dev_err, pad;
@@ -85,8 +86,11 @@ struct scout_plan {
     bool launched = false;
 
     // optional in-stream timing of the scan kernel (key "timing")
+    // a ring of event pairs, one per sign launch, so that a caller can time every launch of a
+    // loop and read the durations after it
     bool timing = false;
-    cudaEvent_t ev_t0 = nullptr, ev_t1 = nullptr;
+    std::vector<cudaEvent_t> ev_t0, ev_t1;
+    uint64_t timed_launches = 0;
 };
 
 namespace {
@@ -166,10 +170,14 @@ int sign_all(scout_plan *p, cudaStream_t stream, scout_sig_t *d_sigs, CertifyOut
     l.variant = p->variant;
     l.uniform_dtype = p->uniform_dtype;
     l.grid = p->grid;
-    if (p->timing) SCOUT_CUDA(cudaEventRecord(p->ev_t0, stream));
+    const size_t slot = p->timing ? (size_t)(p->timed_launches % p->ev_t0.size()) : 0;
+    if (p->timing) SCOUT_CUDA(cudaEventRecord(p->ev_t0[slot], stream));
     int rc = launch_sign_tiles(l, stream);
     if (rc) return rc;
-    if (p->timing) SCOUT_CUDA(cudaEventRecord(p->ev_t1, stream));
+    if (p->timing) {
+        SCOUT_CUDA(cudaEventRecord(p->ev_t1[slot], stream));
+        p->timed_launches += 1;
+    }
     rc = launch_finalize(p->d_chunks, p->chunks.size(), p->R, p->d_recs, p->tiles.size(),
                          p->tile_bytes / ROW_BYTES, d_sigs, zero_out, stream);
     if (rc) return rc;
@@ -416,8 +424,8 @@ int scout_plan_destroy(scout_plan_t *p) {
     if (p->s_copy) cudaStreamDestroy(p->s_copy);
     if (p->s_comp) cudaStreamDestroy(p->s_comp);
     if (p->ev_last) cudaEventDestroy(p->ev_last);
-    if (p->ev_t0) cudaEventDestroy(p->ev_t0);
-    if (p->ev_t1) cudaEventDestroy(p->ev_t1);
+    for (cudaEvent_t e : p->ev_t0) cudaEventDestroy(e);
+    for (cudaEvent_t e : p->ev_t1) cudaEventDestroy(e);
     (void)cudaGetLastError();
     delete p;
     return SCOUT_OK;
@@ -633,11 +641,20 @@ int scout_plan_set(scout_plan_t *p, const char *key, int64_t value) {
         return sign_grid_size(p->variant, p->uniform_dtype, p->device, &p->grid);
     }
     if (!std::strcmp(key, "timing")) {
-        if (value && !p->ev_t0) {
-            SCOUT_CUDA(cudaEventCreate(&p->ev_t0));
-            SCOUT_CUDA(cudaEventCreate(&p->ev_t1));
+        if (value && p->ev_t0.empty()) {
+            try {
+                p->ev_t0.assign(TIMING_RING, nullptr);
+                p->ev_t1.assign(TIMING_RING, nullptr);
+            } catch (const std::bad_alloc &) {
+                return SCOUT_ERR_NOMEM;
+            }
+            for (size_t i = 0; i < TIMING_RING; ++i) {
+                SCOUT_CUDA(cudaEventCreate(&p->ev_t0[i]));
+                SCOUT_CUDA(cudaEventCreate(&p->ev_t1[i]));
+            }
         }
         p->timing = value != 0;
+        p->timed_launches = 0;  // (re)starts the count the two getters below refer to
         return SCOUT_OK;
     }
     if (!std::strcmp(key, "grid")) {
@@ -654,12 +671,33 @@ int scout_plan_get(const scout_plan_t *p, const char *key, int64_t *value) {
     else if (!std::strcmp(key, "variant")) *value = p->variant;
     else if (!std::strcmp(key, "grid")) *value = p->grid;
     else if (!std::strcmp(key, "n_tiles")) *value = (int64_t)p->tiles.size();
+    else if (!std::strcmp(key, "sign_kernels")) *value = 2;     // scan, finalise
+    else if (!std::strcmp(key, "certify_kernels")) *value = 4;  // + vote, certificate chain
     else if (!std::strcmp(key, "last_sign_ns")) {
         // device time of the most recent scan kernel; the stream must have been synchronised
-        if (!p->timing || !p->ev_t0) return SCOUT_ERR_INVALID;
+        if (!p->timing || p->timed_launches == 0) return SCOUT_ERR_INVALID;
+        const size_t slot = (size_t)((p->timed_launches - 1) % TIMING_RING);
         float ms = 0.f;
-        SCOUT_CUDA(cudaEventElapsedTime(&ms, p->ev_t0, p->ev_t1));
+        SCOUT_CUDA(cudaEventElapsedTime(&ms, p->ev_t0[slot], p->ev_t1[slot]));
         *value = (int64_t)((double)ms * 1e6);
+    }
+    else if (!std::strcmp(key, "timed_sign_launches")) {
+        // scan launches the ring still holds (all of them, up to its size) since "timing" was set
+        if (!p->timing) return SCOUT_ERR_INVALID;
+        *value = (int64_t)std::min<uint64_t>(p->timed_launches, TIMING_RING);
+    }
+    else if (!std::strcmp(key, "timed_sign_ns")) {
+        // their total device time; the stream must have been synchronised
+        if (!p->timing) return SCOUT_ERR_INVALID;
+        const uint64_t n = std::min<uint64_t>(p->timed_launches, TIMING_RING);
+        double total_ms = 0.0;
+        for (uint64_t i = 0; i < n; ++i) {
+            const size_t slot = (size_t)((p->timed_launches - 1 - i) % TIMING_RING);
+            float ms = 0.f;
+            SCOUT_CUDA(cudaEventElapsedTime(&ms, p->ev_t0[slot], p->ev_t1[slot]));
+            total_ms += ms;
+        }
+        *value = (int64_t)(total_ms * 1e6);
     }
     else if (!std::strcmp(key, "device_error")) {
         if (int rc = check_device(p)) return rc;

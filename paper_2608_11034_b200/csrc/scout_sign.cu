@@ -43,12 +43,7 @@ constexpr int SIGN_THREADS = 256;
 #ifndef SCOUT_UNROLL
 #define SCOUT_UNROLL 8
 #endif
-#ifndef SCOUT_HASH_FORM
-#define SCOUT_HASH_FORM 0
-#endif
-#ifndef SCOUT_L2_PREFETCH
-#define SCOUT_L2_PREFETCH 0
-#endif
+
 constexpr int UNROLL = SCOUT_UNROLL;
 // bf16: how many of a word-quad's four high halves are widened by bit placement
 // instead of the conversion pipe (see stats_fast).
@@ -254,21 +249,12 @@ __device__ __noinline__ void rescan_classifying(const uint8_t *tile, uint32_t nb
 // h * P lets every product be a 32x32+64 multiply-add (measured: fewest
 // instructions of the forms tried; a 64-bit accumulate costs two issue slots).
 __device__ __forceinline__ void fold_row(uint64_t &h, const uint4 &v, const uint32_t (&m)[4]) {
-#if SCOUT_HASH_FORM == 1
-    // row sum first (independent of h), then one short dependent step on h
-    uint64_t t = (uint64_t)m[0] * v.x;
-    t += (uint64_t)m[1] * v.y;
-    t += (uint64_t)m[2] * v.z;
-    t += (uint64_t)m[3] * v.w;
-    h = h * HASH_P + t;
-#else
     uint64_t t = h * HASH_P;
     t += (uint64_t)m[0] * v.x;
     t += (uint64_t)m[1] * v.y;
     t += (uint64_t)m[2] * v.z;
     t += (uint64_t)m[3] * v.w;
     h = t;
-#endif
 }
 
 // Per-lane state of one tile's scan: the lane's four slot multipliers, its share
@@ -287,6 +273,9 @@ struct TileScan {
         h = 0;
         a = Acc{0.0, 0.0, 0.0, 0.0};
     }
+    // the two halves of a row's work, separately (the cost microbenchmark times each alone)
+    __device__ __forceinline__ void row_hash(const uint4 &v) { fold_row(h, v, m); }
+    __device__ __forceinline__ void row_stats(const uint4 &v) { stats_fast<DT>(v, a); }
     __device__ __forceinline__ void row(const uint4 &v) {
         fold_row(h, v, m);
         stats_fast<DT>(v, a);
@@ -347,12 +336,6 @@ __device__ __forceinline__ void scan_tile(const uint8_t *tile, uint32_t nbytes, 
         uint4 v[UNROLL];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) v[u] = ld_stream16(p + u * ROW_BYTES);
-#if SCOUT_L2_PREFETCH
-        // ask L2 for the next batch while this one is folded
-        if (lane == 0 && b > 1)
-            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p + UNROLL * ROW_BYTES),
-                         "r"((uint32_t)(UNROLL * ROW_BYTES)) : "memory");
-#endif
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) st.row(v[u]);
     }

@@ -106,3 +106,45 @@ def test_three_ranks_gather_and_vote_identically():
     assert [r[1:] for r in res] == [res[0][1:]] * 3
     chunk = (777 * 4) // 65536
     assert res[0][1] == [(chunk, 1)] and res[0][2] == []
+
+
+def _records_worker(rank, world, port, out):
+    """The product's gather step (gloo path: records in host memory) on oracle-signed records."""
+    os.environ.update(RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from oracle import scout_oracle as orc
+    from paper_2608_11034_b200 import dist_c3, dist_util, inputs
+    import helpers as h
+
+    dist_util.init("gloo")
+    w = inputs.workload(2, "clean", 1 / 64)
+    w.R = world
+    _, views = inputs.generate(w)
+    tt = h.oracle_tensor_table(w)
+    n_ch = len(orc.chunk_table(tt, w.chunk_bytes))
+    mine = np.zeros((n_ch, 1), dtype=orc.SIG_DTYPE)
+    orc.sign_replica(tt, [inputs.to_numpy_bytes(v) for v in views[rank]], w.chunk_bytes, mine, 0, 1)
+    mine["hash"][0, 0] ^= rank                      # make the ranks' rows distinguishable
+    local = torch.from_numpy(mine.view(np.uint8).reshape(-1).copy())
+    table = dist_c3.gather_records(local).numpy().view(orc.SIG_DTYPE).reshape(world, n_ch)
+    out.put((rank, [int(x) for x in table["hash"][:, 0]], table[:, 1:].tobytes() == np.tile(mine[1:, 0], (world, 1)).tobytes()))
+    dist_util.barrier()
+    dist.destroy_process_group()
+
+
+def test_gather_records_is_rank_major_on_every_rank():
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_records_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(out.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert res[0][1] == res[1][1] and res[0][1][0] ^ res[0][1][1] == 1     # row r is rank r's, everywhere
+    assert res[0][2] and res[1][2]
