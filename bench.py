@@ -350,6 +350,38 @@ def run_config(cfg, args, rank, world, local, headline):
     roofline["read_probe_gbs"] = probe
     roofline["frac_of_read_probe"] = achieved / probe
 
+    one_launch = None
+    if small and w.R >= 2:
+        # the whole path as ONE kernel: scout_certify_launch enqueues it, scout_certify_collect
+        # (outside the event pair) waits for the report the kernel wrote to pinned host memory
+        def timed(fn_launch, fn_after, flush_between):
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                   for _ in range(args.steps)]
+            for _ in range(3):
+                fn_launch(); fn_after()
+            torch.cuda.synchronize()
+            for i, (a0, a1) in enumerate(evs):
+                if flush_between:
+                    flush.fill_(i & 255)
+                a0.record(); fn_launch(); a1.record(); fn_after()
+            torch.cuda.synchronize()
+            return sum(a0.elapsed_time(a1) for a0, a1 in evs) / args.steps
+        one_launch = {"call": "scout_certify_launch (+ scout_certify_collect outside the timed pair)"}
+        for name, fused in (("one_kernel", 1), ("kernel_per_stage", 0)):
+            binding.scout_plan_set(plan.handle, "fused", fused)
+            cold = timed(plan.certify_launch, plan.certify_collect, True)
+            warm1 = timed(plan.certify_launch, plan.certify_collect, False)
+            t0 = time.perf_counter()
+            for _ in range(args.steps):
+                rep = plan.certify()
+            wall = (time.perf_counter() - t0) / args.steps
+            assert rep["outliers"] == want
+            one_launch[name] = {"kernels_per_step": binding.scout_plan_get(plan.handle, "certify_kernels"),
+                                "ms_per_step_l2_cold": cold, "ms_per_step_l2_warm": warm1,
+                                "value_l2_cold": total_bytes / (cold * 1e-3) / 1e9,
+                                "scout_certify_wall_ms_l2_warm": wall * 1e3}
+        binding.scout_plan_set(plan.handle, "fused", -1)
+
     warm = None
     if small:   # the same steps with the replicas left in L2 (no flush between steps)
         evw = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
@@ -378,6 +410,7 @@ def run_config(cfg, args, rank, world, local, headline):
         "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
         "frac_of_measured_copy": value / world / peak,
         "verified": True, "verdict": verdict, "clocks": clocks, "roofline": roofline, "l2_warm": warm,
+        "one_launch": one_launch,
     }
 
     # ---- end to end: replicas in pinned host memory, copies inside the timed region
@@ -515,6 +548,7 @@ def main():
         "verified": head["verified"], "verdict": head["verdict"],
         "gpu_launches": head["launch"]["kernels_per_step"] * args.steps,
         "clocks": head["clocks"], "roofline": head["roofline"], "l2_warm": head["l2_warm"],
+        "one_launch": head["one_launch"],
         "e2e": head["e2e"], "cpu_baseline": head["cpu_baseline"],
     }
 

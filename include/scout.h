@@ -190,6 +190,19 @@ SCOUT_API int scout_certify(scout_plan_t *plan, void *stream, scout_report_t *re
                   scout_outlier_t *h_outliers /*host*/, uint64_t outlier_cap,
                   uint64_t *h_undecided /*host*/, uint64_t undecided_cap);
 
+/* The same run in two halves, for callers that must not block where the check is
+ * enqueued (C3 runs in the progress path of a training step, Sec. 9): the first
+ * call enqueues everything on `stream` and returns; the second waits for it and
+ * fills the report and the sorted lists exactly as scout_certify does.  The
+ * lists are cut at the capacities given to the first call (the second call's
+ * capacities may be smaller, not larger).  One run may be in flight per plan:
+ * a second launch, or a scout_certify, before the collect is SCOUT_ERR_INVALID. */
+SCOUT_API int scout_certify_launch(scout_plan_t *plan, void *stream, uint64_t outlier_cap,
+                                   uint64_t undecided_cap);
+SCOUT_API int scout_certify_collect(scout_plan_t *plan, scout_report_t *report /*host*/,
+                                    scout_outlier_t *h_outliers /*host*/, uint64_t outlier_cap,
+                                    uint64_t *h_undecided /*host*/, uint64_t undecided_cap);
+
 /* After scout_certify: device pointers to the plan-owned results of that run
  * (valid until the next certify or destroy).  Any output may be NULL. */
 SCOUT_API int scout_plan_results(const scout_plan_t *plan, const scout_sig_t **d_sigs,
@@ -259,6 +272,16 @@ SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/)
  *                     consumer warps share them (needs tile_bytes <= 32768);
  *                     3 = read-only probe (measures the memory system only: the
  *                     records it leaves are NOT signatures)
+ *   set "fused"       with the default scan (variant 0) and R <= 64 a call can run as
+ *                     ONE kernel: the warp that stores the last tile record of a chunk
+ *                     finalises it (scout_sign_chunks), and for scout_certify also votes
+ *                     it and folds it into the certificate chain; the warp that folds the
+ *                     last chunk writes the report block to pinned host memory.
+ *                     1: always; 0: never (one kernel per stage: scan, finalise, vote,
+ *                     certificate - the form scout_certify_host always uses); -1
+ *                     (default): where it is the faster form - scout_certify always;
+ *                     scout_sign_chunks for plans of 1 GB and more whose tensors are all
+ *                     fp32 or all bf16
  *   set "grid"        CTAs of the scan kernel
  *   set "timing"      1: record a pair of CUDA events around every scan kernel on
  *                     the caller's stream (a ring of 256 pairs); setting it again

@@ -77,6 +77,8 @@ def lib():
             "scout_consensus_vote": (C.c_int, [u32, u64, vp, vp, vp, vp, u64, vp, u64, vp, vp]),
             "scout_consensus_vote_wide": (C.c_int, [u32, u64, vp, u64, u64, vp, vp, vp, u64, vp, u64, vp, vp]),
             "scout_certify": (C.c_int, [vp, vp, vp, vp, u64, vp, u64]),
+            "scout_certify_launch": (C.c_int, [vp, vp, u64, u64]),
+            "scout_certify_collect": (C.c_int, [vp, vp, vp, u64, vp, u64]),
             "scout_plan_results": (C.c_int, [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)]),
             "scout_plan_replica_bad_counts": (C.c_int, [vp, vp]),
             "scout_rollup_tensors": (C.c_int, [vp, vp, vp, vp]),
@@ -209,6 +211,18 @@ def scout_certify(plan: int, stream: int, outlier_cap: int = 4096, undecided_cap
     """-> dict(report, outliers [(chunk, replica)] sorted, undecided sorted, rc)"""
     return _certify_common(lib().scout_certify, "scout_certify", plan, stream, outlier_cap,
                            undecided_cap)
+
+
+def scout_certify_launch(plan: int, stream: int, outlier_cap: int = 4096, undecided_cap: int = 4096) -> None:
+    """Enqueue one certify run on `stream` and return; scout_certify_collect finishes it."""
+    _check(lib().scout_certify_launch(plan, stream, outlier_cap, undecided_cap), "scout_certify_launch")
+
+
+def scout_certify_collect(plan: int, outlier_cap: int = 4096, undecided_cap: int = 4096):
+    """Wait for the launched run.  -> the same dict as scout_certify."""
+    fn = lib().scout_certify_collect
+    return _certify_common(lambda pl, _unused, *rest: fn(pl, *rest), "scout_certify_collect", plan, None,
+                           outlier_cap, undecided_cap)
 
 
 def scout_certify_host(plan: int, h_ptrs: Sequence[int], outlier_cap: int = 4096,
@@ -455,3 +469,11 @@ class Plan:
     def certify(self, outlier_cap: int = 4096, undecided_cap: int = 4096, stream: Optional[int] = None):
         s = self._torch.cuda.current_stream().cuda_stream if stream is None else stream
         return scout_certify(self.handle, s, outlier_cap, undecided_cap)
+
+    def certify_launch(self, outlier_cap: int = 4096, undecided_cap: int = 4096,
+                       stream: Optional[int] = None) -> None:
+        s = self._torch.cuda.current_stream().cuda_stream if stream is None else stream
+        scout_certify_launch(self.handle, s, outlier_cap, undecided_cap)
+
+    def certify_collect(self, outlier_cap: int = 4096, undecided_cap: int = 4096):
+        return scout_certify_collect(self.handle, outlier_cap, undecided_cap)

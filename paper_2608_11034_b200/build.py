@@ -23,7 +23,7 @@ def _nvcc() -> str:
 
 def sources():
     srcs = [os.path.join(CSRC, s) for s in SOURCES]
-    deps = srcs + [os.path.join(CSRC, "scout_internal.h")] + \
+    deps = srcs + [os.path.join(CSRC, h) for h in ("scout_internal.h", "scout_vote_device.cuh")] + \
         [os.path.join(ROOT, "include", h) for h in sorted(os.listdir(os.path.join(ROOT, "include")))]
     return srcs, deps
 

@@ -34,15 +34,7 @@ static uint32_t dtype_size(uint32_t d) {
 
 using namespace scout;
 
-// Pinned landing area of scout_certify's device-to-host copies.
-constexpr uint64_t CERTIFY_HEAD = 64;
 constexpr size_t TIMING_RING = 256;  // event pairs kept for the "timing" knob
-struct CertifyHost {
-    CertifyOut out;
-    uint32_t dev_err, pad;
-    scout_outlier_t outliers[CERTIFY_HEAD];
-    uint64_t undecided[CERTIFY_HEAD];
-};
 
 struct scout_plan {
     uint32_t R = 0;
@@ -73,6 +65,21 @@ struct scout_plan {
     CertifyOut *d_out = nullptr;
     CertifyHost *h_out = nullptr;  // pinned
     bool have_results = false;
+
+    // one-launch path (certify_tiles): per-chunk tickets, launch stamps, chain state
+    int fused = -1;               // key "fused": 1 always, 0 never, -1 where it is the faster form (see
+                                  // use_fused); only the default scan (variant 0) has a one-launch form
+    uint64_t total_bytes = 0;     // R * bytes per replica
+    int fused_grid = 0;
+    uint32_t *d_tickets = nullptr, *d_done = nullptr;
+    ChainState *d_chain = nullptr;
+    unsigned long long *d_work = nullptr;
+    CertifyHost *h_out_dev = nullptr;  // device-side address of h_out
+    uint32_t epoch = 0;
+    bool out_dirty = false;       // d_out was left non-zero by the multi-kernel path
+    bool pending = false;         // a certify was launched and not collected yet
+    cudaStream_t pending_stream = nullptr;
+    uint64_t pending_ocap = 0, pending_ucap = 0;
 
     // host-replica staging
     uint8_t *d_stage[2] = {nullptr, nullptr};
@@ -137,6 +144,7 @@ void build_tiles(scout_plan *p) {
             p->tiles.push_back(td);
         }
         cd.ntiles = n;
+        for (uint32_t j = 0; j < n; ++j) p->tiles[cd.tile0 + j].chunk_tiles = n;
     }
 }
 
@@ -153,7 +161,86 @@ int upload_tables(scout_plan *p) {
     return SCOUT_OK;
 }
 
+// Is this call made as one launch?  Measured on B200.  scout_certify: always - one kernel
+// instead of four plus the copies is faster at every size (12.6 MB: 34 against 42 us on the
+// device, 51 against 67 us per call; 36 GB: +1 %), and from a few thousand chunks on it also
+// hides the sequential certificate chain behind the scan.  scout_sign_chunks alone: only for
+// plans of 1 GB and more whose tensors are all fp32 or all bf16.  Below that the scan and the
+// finalise kernel launched back to back (programmatic dependent launch) are faster, because the
+// ticket and the finalisation by the last warp add L2 round trips of about a microsecond each
+// to a kernel that runs for tens of microseconds; and the kernel that reads the dtype from the
+// tile table spills registers in its one-launch form (-2 % on 10,000 mixed tensors).
+bool use_fused(const scout_plan *p, bool certify) {
+    if (p->variant != 0 || p->R > 64 || !p->d_tickets || p->fused == 0) return false;
+    if (p->fused > 0 || certify) return true;
+    return p->total_bytes >= (1ull << 30) &&
+           (p->uniform_dtype == SCOUT_DT_F32 || p->uniform_dtype == SCOUT_DT_BF16);
+}
+
+void fill_sign_launch(const scout_plan *p, SignLaunch &l) {
+    l.tiles = p->d_tiles;
+    l.tile_begin = 0;
+    l.n_tiles = p->tiles.size();
+    l.tiles_per_replica = p->tiles.size();
+    l.replica_begin = 0;
+    l.n_replicas = p->R;
+    l.ptrs = (const uint8_t *const *)p->d_ptrs;
+    l.T = p->T;
+    l.stage = nullptr;
+    l.slice_begin = 0;
+    l.recs = p->d_recs;
+    l.error = p->d_error;
+    l.variant = p->variant;
+    l.uniform_dtype = p->uniform_dtype;
+    l.grid = p->grid;
+}
+
+// One kernel: scan + finalise (certify == false), or the whole certify path.  The timing
+// events bracket that kernel.
+int launch_one_kernel(scout_plan *p, cudaStream_t stream, scout_sig_t *d_sigs, bool certify,
+                      uint64_t outlier_cap, uint64_t undecided_cap) {
+    FusedLaunch f;
+    std::memset(&f, 0, sizeof(f));
+    fill_sign_launch(p, f.sign);
+    f.sign.grid = p->fused_grid;
+    f.chunks = p->d_chunks;
+    f.C = p->chunks.size();
+    f.R = p->R;
+    f.tile_rows = p->tile_bytes / ROW_BYTES;
+    f.sigs = d_sigs;
+    f.mode = certify ? 1 : 0;
+    f.tickets = p->d_tickets;
+    f.work = p->d_work;
+    uint32_t max_tiles = 0;
+    for (const ChunkDesc &cd : p->chunks) max_tiles = std::max(max_tiles, cd.ntiles);
+    f.one_level = (uint64_t)max_tiles * p->R <= 64 ? 1u : 0u;
+    if (++p->epoch == 0) p->epoch = 1;  // 0 is the stamp of "never"
+    f.epoch = p->epoch;
+    if (certify) {
+        if (p->out_dirty) {
+            SCOUT_CUDA(cudaMemsetAsync(p->d_out, 0, sizeof(CertifyOut), stream));
+            p->out_dirty = false;
+        }
+        f.vote = VoteSinks{p->d_status, p->d_bitmap, p->d_majority, p->d_outliers, outlier_cap,
+                           p->d_undecided, undecided_cap, p->d_out->counts, p->d_out};
+        f.out = p->d_out;
+        f.done = p->d_done;
+        f.chain = p->d_chain;
+        f.host = p->h_out_dev;
+    }
+    const size_t slot = p->timing ? (size_t)(p->timed_launches % p->ev_t0.size()) : 0;
+    if (p->timing) SCOUT_CUDA(cudaEventRecord(p->ev_t0[slot], stream));
+    int rc = launch_fused(f, stream);
+    if (rc) return rc;
+    if (p->timing) {
+        SCOUT_CUDA(cudaEventRecord(p->ev_t1[slot], stream));
+        p->timed_launches += 1;
+    }
+    return mark_launched(p, stream);
+}
+
 int sign_all(scout_plan *p, cudaStream_t stream, scout_sig_t *d_sigs, CertifyOut *zero_out = nullptr) {
+    if (use_fused(p, false) && !zero_out) return launch_one_kernel(p, stream, d_sigs, false, 0, 0);
     SignLaunch l;
     l.tiles = p->d_tiles;
     l.tile_begin = 0;
@@ -192,7 +279,9 @@ int ensure_certify_buffers(scout_plan *p, uint64_t outlier_cap, uint64_t undecid
         SCOUT_CUDA(cudaMalloc(&p->d_bitmap, C * sizeof(uint64_t)));
         SCOUT_CUDA(cudaMalloc(&p->d_majority, C * sizeof(uint64_t)));
         SCOUT_CUDA(cudaMalloc(&p->d_out, sizeof(CertifyOut)));
-        SCOUT_CUDA(cudaMallocHost(&p->h_out, sizeof(CertifyHost)));
+        SCOUT_CUDA(cudaMemset(p->d_out, 0, sizeof(CertifyOut)));
+        SCOUT_CUDA(cudaHostAlloc(&p->h_out, sizeof(CertifyHost), cudaHostAllocMapped));
+        SCOUT_CUDA(cudaHostGetDevicePointer((void **)&p->h_out_dev, p->h_out, 0));
     }
     if (!p->d_outliers || outlier_cap > p->outlier_cap) {
         if (p->d_outliers) cudaFree(p->d_outliers);
@@ -209,18 +298,17 @@ int ensure_certify_buffers(scout_plan *p, uint64_t outlier_cap, uint64_t undecid
     return SCOUT_OK;
 }
 
-// vote + certificate + copy-back + host canonicalisation, after d_sigs is ready on `stream`
-int vote_and_report(scout_plan *p, cudaStream_t stream, scout_report_t *report,
-                    scout_outlier_t *h_outliers, uint64_t outlier_cap, uint64_t *h_undecided,
-                    uint64_t undecided_cap) {
+// Multi-kernel path: vote + certificate + speculative copies of the report block, after
+// d_sigs is ready on `stream` (the finalise kernel that precedes this cleared d_out).
+int enqueue_vote_and_copies(scout_plan *p, cudaStream_t stream, uint64_t outlier_cap, uint64_t undecided_cap) {
     const uint64_t C = p->chunks.size();
-    // the finalise kernel that precedes this on the stream cleared d_out
     int rc = launch_vote(p->R, C, p->d_sigs, p->d_status, p->d_bitmap, p->d_outliers, outlier_cap,
                          p->d_undecided, undecided_cap, p->d_out->counts, p->d_majority, p->d_out, true,
                          stream);
     if (rc) return rc;
     rc = launch_certificate(C, p->d_majority, p->d_out, stream);
     if (rc) return rc;
+    p->out_dirty = true;
     // One round trip in the common case: the counters, the error flag and the head of
     // both lists are copied speculatively; longer lists need a second copy.
     CertifyHost *hh = p->h_out;
@@ -234,7 +322,19 @@ int vote_and_report(scout_plan *p, cudaStream_t stream, scout_report_t *report,
     if (head_und)
         SCOUT_CUDA(cudaMemcpyAsync(hh->undecided, p->d_undecided, head_und * sizeof(uint64_t),
                                    cudaMemcpyDeviceToHost, stream));
+    return SCOUT_OK;
+}
+
+// Waits for the launched certify and turns the report block (in pinned host memory, written
+// by copies or by the one-launch kernel itself) into the caller's report and canonical lists.
+int collect_report(scout_plan *p, cudaStream_t stream, scout_report_t *report,
+                   scout_outlier_t *h_outliers, uint64_t outlier_cap, uint64_t *h_undecided,
+                   uint64_t undecided_cap) {
     SCOUT_CUDA(cudaStreamSynchronize(stream));
+    p->pending = false;
+    CertifyHost *hh = p->h_out;
+    const uint64_t head_out = std::min<uint64_t>(outlier_cap, CERTIFY_HEAD);
+    const uint64_t head_und = std::min<uint64_t>(undecided_cap, CERTIFY_HEAD);
     const CertifyOut &o = hh->out;
     const uint64_t n_out = std::min<uint64_t>(o.counts[4], outlier_cap);
     const uint64_t n_und = std::min<uint64_t>(o.counts[5], undecided_cap);
@@ -273,6 +373,32 @@ int vote_and_report(scout_plan *p, cudaStream_t stream, scout_report_t *report,
         return SCOUT_ERR_CUDA;
     }
     return (o.counts[4] > outlier_cap || o.counts[5] > undecided_cap) ? SCOUT_ERR_TRUNCATED : SCOUT_OK;
+}
+
+int vote_and_report(scout_plan *p, cudaStream_t stream, scout_report_t *report,
+                    scout_outlier_t *h_outliers, uint64_t outlier_cap, uint64_t *h_undecided,
+                    uint64_t undecided_cap) {
+    int rc = enqueue_vote_and_copies(p, stream, outlier_cap, undecided_cap);
+    if (rc) return rc;
+    return collect_report(p, stream, report, h_outliers, outlier_cap, h_undecided, undecided_cap);
+}
+
+// Enqueues one certify run on `stream` (either path); collect_report() finishes it.
+int certify_enqueue(scout_plan *p, cudaStream_t stream, uint64_t outlier_cap, uint64_t undecided_cap) {
+    int rc = ensure_certify_buffers(p, outlier_cap, undecided_cap);
+    if (rc) return rc;
+    if (use_fused(p, true)) {
+        rc = launch_one_kernel(p, stream, p->d_sigs, true, outlier_cap, undecided_cap);
+    } else {
+        if ((rc = sign_all(p, stream, p->d_sigs, p->d_out))) return rc;
+        rc = enqueue_vote_and_copies(p, stream, outlier_cap, undecided_cap);
+    }
+    if (rc) return rc;
+    p->pending = true;
+    p->pending_stream = stream;
+    p->pending_ocap = outlier_cap;
+    p->pending_ucap = undecided_cap;
+    return SCOUT_OK;
 }
 
 }  // namespace
@@ -331,6 +457,7 @@ int scout_plan_create(uint32_t R, uint64_t T, const scout_tensor_t *tensors, uin
             delete p;
             return SCOUT_ERR_UNSUPPORTED;
         }
+        p->total_bytes = total * R;
         p->tile_bytes = auto_tile_bytes(total * R);
         build_tiles(p);
     } catch (const std::bad_alloc &) {
@@ -348,6 +475,23 @@ int scout_plan_create(uint32_t R, uint64_t T, const scout_tensor_t *tensors, uin
             rc = SCOUT_ERR_NOMEM;
             break;
         }
+        const size_t nc = p->chunks.size();
+        const size_t n_tickets = nc * R + nc;  // one per (chunk, replica), then one per chunk
+        if (cudaMalloc(&p->d_tickets, n_tickets * sizeof(uint32_t)) != cudaSuccess ||
+            cudaMalloc(&p->d_done, nc * sizeof(uint32_t)) != cudaSuccess ||
+            cudaMalloc(&p->d_chain, sizeof(ChainState)) != cudaSuccess ||
+            cudaMalloc(&p->d_work, 2 * sizeof(unsigned long long)) != cudaSuccess) {
+            rc = SCOUT_ERR_NOMEM;
+            break;
+        }
+        if (cudaMemset(p->d_tickets, 0, n_tickets * sizeof(uint32_t)) != cudaSuccess ||
+            cudaMemset(p->d_done, 0, nc * sizeof(uint32_t)) != cudaSuccess ||
+            cudaMemset(p->d_chain, 0, sizeof(ChainState)) != cudaSuccess ||
+            cudaMemset(p->d_work, 0, 2 * sizeof(unsigned long long)) != cudaSuccess) {
+            rc = SCOUT_ERR_CUDA;
+            break;
+        }
+        if ((rc = fused_grid_size(p->uniform_dtype, p->device, &p->fused_grid))) break;
         if (cudaMemset(p->d_error, 0, sizeof(uint32_t)) != cudaSuccess ||
             cudaEventCreateWithFlags(&p->ev_last, cudaEventDisableTiming) != cudaSuccess) {
             rc = SCOUT_ERR_CUDA;
@@ -408,6 +552,10 @@ int scout_plan_destroy(scout_plan_t *p) {
     cudaFree((void *)p->d_ptrs);
     cudaFree(p->d_recs);
     cudaFree(p->d_error);
+    cudaFree(p->d_tickets);
+    cudaFree(p->d_done);
+    cudaFree(p->d_chain);
+    cudaFree(p->d_work);
     cudaFree(p->d_sigs);
     cudaFree(p->d_status);
     cudaFree(p->d_bitmap);
@@ -463,17 +611,37 @@ int scout_consensus_vote_wide(uint32_t R, uint64_t C, const scout_sig_t *d_sigs,
                             outlier_cap, d_undecided, undecided_cap, d_counts, (cudaStream_t)stream);
 }
 
+int scout_certify_launch(scout_plan_t *p, void *stream, uint64_t outlier_cap, uint64_t undecided_cap) {
+    if (!p || !p->bound || p->R < 2) return SCOUT_ERR_INVALID;
+    if (p->R > 64) return SCOUT_ERR_UNSUPPORTED;
+    if (p->pending) return SCOUT_ERR_INVALID;  // one run in flight per plan: collect it first
+    int rc = check_device(p);
+    if (rc) return rc;
+    return certify_enqueue(p, (cudaStream_t)stream, outlier_cap, undecided_cap);
+}
+
+int scout_certify_collect(scout_plan_t *p, scout_report_t *report, scout_outlier_t *h_outliers,
+                          uint64_t outlier_cap, uint64_t *h_undecided, uint64_t undecided_cap) {
+    if (!p || !report || !p->pending) return SCOUT_ERR_INVALID;
+    if ((outlier_cap && !h_outliers) || (undecided_cap && !h_undecided)) return SCOUT_ERR_INVALID;
+    if (outlier_cap > p->pending_ocap || undecided_cap > p->pending_ucap) return SCOUT_ERR_INVALID;
+    int rc = check_device(p);
+    if (rc) return rc;
+    // the device lists were cut at the capacities given at launch
+    return collect_report(p, p->pending_stream, report, h_outliers, outlier_cap, h_undecided, undecided_cap);
+}
+
 int scout_certify(scout_plan_t *p, void *stream, scout_report_t *report, scout_outlier_t *h_outliers,
                   uint64_t outlier_cap, uint64_t *h_undecided, uint64_t undecided_cap) {
     if (!p || !report || !p->bound || p->R < 2) return SCOUT_ERR_INVALID;
     if (p->R > 64) return SCOUT_ERR_UNSUPPORTED;
     if ((outlier_cap && !h_outliers) || (undecided_cap && !h_undecided)) return SCOUT_ERR_INVALID;
+    if (p->pending) return SCOUT_ERR_INVALID;
     int rc = check_device(p);
     if (rc) return rc;
-    if ((rc = ensure_certify_buffers(p, outlier_cap, undecided_cap))) return rc;
     cudaStream_t s = (cudaStream_t)stream;
-    if ((rc = sign_all(p, s, p->d_sigs, p->d_out))) return rc;
-    return vote_and_report(p, s, report, h_outliers, outlier_cap, h_undecided, undecided_cap);
+    if ((rc = certify_enqueue(p, s, outlier_cap, undecided_cap))) return rc;
+    return collect_report(p, s, report, h_outliers, outlier_cap, h_undecided, undecided_cap);
 }
 
 int scout_certify_host(scout_plan_t *p, const void *const *h_ptrs, scout_report_t *report,
@@ -634,6 +802,11 @@ int scout_plan_set(scout_plan_t *p, const char *key, int64_t value) {
         }
         return upload_tables(p);
     }
+    if (!std::strcmp(key, "fused")) {
+        if (value < -1 || value > 1) return SCOUT_ERR_INVALID;
+        p->fused = (int)value;
+        return SCOUT_OK;
+    }
     if (!std::strcmp(key, "variant")) {
         if (value < 0 || value > 4) return SCOUT_ERR_INVALID;
         if (value == 4 && p->tile_bytes > 32768) return SCOUT_ERR_INVALID;  // a tile must fit one stage
@@ -671,8 +844,9 @@ int scout_plan_get(const scout_plan_t *p, const char *key, int64_t *value) {
     else if (!std::strcmp(key, "variant")) *value = p->variant;
     else if (!std::strcmp(key, "grid")) *value = p->grid;
     else if (!std::strcmp(key, "n_tiles")) *value = (int64_t)p->tiles.size();
-    else if (!std::strcmp(key, "sign_kernels")) *value = 2;     // scan, finalise
-    else if (!std::strcmp(key, "certify_kernels")) *value = 4;  // + vote, certificate chain
+    else if (!std::strcmp(key, "fused")) *value = p->fused;
+    else if (!std::strcmp(key, "sign_kernels")) *value = use_fused(p, false) ? 1 : 2;    // scan, finalise
+    else if (!std::strcmp(key, "certify_kernels")) *value = use_fused(p, true) ? 1 : 4;  // + vote, certificate chain
     else if (!std::strcmp(key, "last_sign_ns")) {
         // device time of the most recent scan kernel; the stream must have been synchronised
         if (!p->timing || p->timed_launches == 0) return SCOUT_ERR_INVALID;

@@ -40,10 +40,9 @@ __host__ __device__ inline uint64_t mix64(uint64_t z) {
 // P^e mod 2^64 by square and multiply.
 __host__ __device__ inline uint64_t pow_p(uint64_t e) {
     uint64_t r = 1, b = HASH_P;
-    while (e) {
-        if (e & 1) r *= b;
+    for (; e; e >>= 1) {  // a select, not a branch: the lanes of a warp come with different exponents
+        r *= (e & 1) ? b : 1ull;
         b *= b;
-        e >>= 1;
     }
     return r;
 }
@@ -65,7 +64,8 @@ struct TileDesc {
     uint32_t tensor;  // tensor index
     uint32_t nbytes;  // bytes in this tile (<= tile_bytes; only a chunk's last tile is short)
     uint32_t chunk;   // global chunk id
-    uint32_t dtype;   // SCOUT_DT_*
+    uint32_t dtype : 8;         // SCOUT_DT_*
+    uint32_t chunk_tiles : 24;  // tiles of this tile's chunk (at most 2^19: 1 GiB in 2 KiB tiles)
 };
 static_assert(sizeof(TileDesc) == 32, "TileDesc layout");
 
@@ -96,6 +96,38 @@ struct CertifyOut {
     uint64_t union_bitmap;
     uint64_t certificate;
     uint64_t replica_bad[64];
+};
+
+// What scout_certify brings back to the host in one piece: the counters, the device
+// error flag and the first CERTIFY_HEAD entries of both lists.  The one-launch certify
+// kernel writes it straight into pinned host memory; the multi-kernel path copies it.
+constexpr uint64_t CERTIFY_HEAD = 64;
+struct CertifyHost {
+    CertifyOut out;
+    uint32_t dev_err, pad;
+    scout_outlier_t outliers[CERTIFY_HEAD];
+    uint64_t undecided[CERTIFY_HEAD];
+};
+
+// Where a vote leaves its results (all device memory).
+struct VoteSinks {
+    uint8_t *status;            // [C] or null
+    uint64_t *bitmap;           // [C] or null
+    uint64_t *majority;         // [C] or null: e* of every decided chunk (0 if Inconclusive)
+    scout_outlier_t *outliers;  // list, capacity outlier_cap
+    uint64_t outlier_cap;
+    uint64_t *undecided;        // list, capacity undecided_cap
+    uint64_t undecided_cap;
+    uint64_t *counts;           // [6]: the two list counters (4, 5) are advanced by vote_chunk()
+    CertifyOut *cert;           // per-replica bad-chunk counts, or null
+};
+
+// Progress of the certificate chain inside a one-launch certify (device, zero between launches).
+struct ChainState {
+    uint32_t lock;  // 1 while a warp is folding chunks into the chain
+    uint32_t pad;
+    uint64_t next;  // chunks folded so far
+    uint64_t a;     // chain value after `next` chunks
 };
 
 // ---- error plumbing ------------------------------------------------------------
@@ -153,6 +185,29 @@ struct SignLaunch {
     int grid;                     // CTAs to launch
 };
 int launch_sign_tiles(const SignLaunch &a, cudaStream_t stream);
+
+// One launch for scan + finalise (mode 0), or scan + finalise + vote + certificate +
+// report (mode 1): see certify_tiles in scout_sign.cu.
+struct FusedLaunch {
+    SignLaunch sign;            // the whole plan: tile_begin 0, every tile, every replica, ptrs set
+    const ChunkDesc *chunks;    // device [C]
+    uint64_t C;
+    uint32_t R;
+    uint32_t tile_rows;
+    scout_sig_t *sigs;          // device [C][R]
+    int mode;                   // 0 sign only, 1 certify
+    VoteSinks vote;             // mode 1
+    CertifyOut *out;            // mode 1: device counters, zero on entry; left zero on exit
+    uint32_t *tickets;          // device [C*R + C], zero on entry; left zero on exit
+    uint32_t *done;             // mode 1: device [C] launch stamps
+    uint32_t epoch;             // this launch's stamp (never 0); successive launches alternate its parity
+    unsigned long long *work;   // device [2]: dynamic work counters, zero on entry (see certify_tiles)
+    uint32_t one_level;         // 1: every chunk has at most 64 (tile, replica) items: chunk tickets only
+    ChainState *chain;          // mode 1: zero on entry; left zero on exit
+    CertifyHost *host;          // mode 1: pinned host memory (device-accessible address)
+};
+int launch_fused(const FusedLaunch &l, cudaStream_t stream);
+int fused_grid_size(int uniform_dtype, int device, int *grid);
 int sign_grid_size(int variant, int uniform_dtype, int device, int *grid);
 int launch_bounded_wait_selftest(uint64_t limit_ns, uint64_t *d_out, cudaStream_t stream);
 

@@ -21,7 +21,10 @@
 #include <mutex>
 #include <type_traits>
 
+#include <cstddef>
+
 #include "scout_internal.h"
+#include "scout_vote_device.cuh"
 
 namespace scout {
 namespace {
@@ -43,6 +46,7 @@ constexpr int SIGN_THREADS = 256;
 #ifndef SCOUT_UNROLL
 #define SCOUT_UNROLL 8
 #endif
+
 
 constexpr int UNROLL = SCOUT_UNROLL;
 // bf16: how many of a word-quad's four high halves are widened by bit placement
@@ -1003,27 +1007,52 @@ constexpr int FIN_THREADS = 128;
 // One warp turns the tile records of one (chunk, replica) into its signature record
 // (valid in lane 0).  tr: the chunk's nt records in order; every tile but the last
 // has tile_rows rows; p_stride = P^(32 * tile_rows).
+// A tile record as another SM wrote it: read through L2.  (L1 is not coherent, and a
+// 128-byte line holds four records, so a line fetched while a neighbouring chunk was being
+// finalised may hold records that had not been written yet.)
+__device__ __forceinline__ TileRec load_record(const TileRec *p) {
+    const uint4 lo = __ldcg(reinterpret_cast<const uint4 *>(p));
+    const uint4 hi = __ldcg(reinterpret_cast<const uint4 *>(p) + 1);
+    TileRec r;
+    r.h = ((uint64_t)lo.y << 32) | lo.x;
+    r.sum = __hiloint2double((int)lo.w, (int)lo.z);
+    r.sumsq = __hiloint2double((int)hi.y, (int)hi.x);
+    r.nan_count = hi.z;
+    r.inf_count = hi.w;
+    return r;
+}
+
+// Weight of a lane's share in combine_tiles: P^(rows that follow the last full tile the
+// lane walks).  It depends on the chunk's geometry only, so it is computed once per chunk
+// and reused for every replica.
+__device__ __forceinline__ uint64_t combine_weight(uint32_t nt, uint64_t nbytes, uint32_t tile_rows,
+                                                   uint32_t lane) {
+    const uint32_t n_full = nt - 1;  // every tile but the chunk's last has tile_rows rows
+    if (lane >= n_full) return 1ull;
+    const uint64_t rows_total = (nbytes + ROW_BYTES - 1) / ROW_BYTES;
+    const uint64_t rows_last = rows_total - (uint64_t)n_full * tile_rows;
+    const uint32_t last_t = lane + ((n_full - 1 - lane) / 32u) * 32u;
+    return pow_p(rows_last + (uint64_t)tile_rows * (n_full - 1 - last_t));
+}
+
 __device__ __forceinline__ scout_sig_t combine_tiles(const TileRec *tr, uint32_t nt, uint64_t nbytes,
                                                      uint64_t k, uint32_t dtype, uint64_t meta,
-                                                     uint32_t tile_rows, uint64_t p_stride, uint32_t lane) {
-    const uint64_t rows_total = (nbytes + ROW_BYTES - 1) / ROW_BYTES;
-    const uint64_t rows_last = rows_total - (uint64_t)(nt - 1) * tile_rows;
+                                                     uint64_t p_stride, uint64_t weight, uint32_t lane) {
     uint64_t h = 0;
     double s = 0.0, q = 0.0;
-    uint32_t nan_count = 0, inf_count = 0, last_t = 0;
-    const uint32_t n_full = nt - 1;  // every tile but the chunk's last has tile_rows rows
+    uint32_t nan_count = 0, inf_count = 0;
+    const uint32_t n_full = nt - 1;
     for (uint32_t t = lane; t < n_full; t += 32) {
-        const TileRec x = tr[t];
+        const TileRec x = load_record(tr + t);
         h = h * p_stride + x.h;
         s += x.sum;
         q += x.sumsq;
         nan_count += x.nan_count;
         inf_count += x.inf_count;
-        last_t = t;
     }
-    if (lane < n_full) h *= pow_p(rows_last + (uint64_t)tile_rows * (n_full - 1 - last_t));
+    if (lane < n_full) h *= weight;
     if (lane == (n_full & 31u)) {  // the last (possibly short) tile: nothing follows it
-        const TileRec x = tr[n_full];
+        const TileRec x = load_record(tr + n_full);
         h += x.h;
         s += x.sum;
         q += x.sumsq;
@@ -1047,6 +1076,41 @@ __device__ __forceinline__ scout_sig_t combine_tiles(const TileRec *tr, uint32_t
     return o;
 }
 
+// The same combine for a chunk of at most 32 tiles (lane t holds tile t), four replicas
+// at a time: their record loads are independent, so they are in flight together.  The
+// arithmetic and its order are those of combine_tiles, so the records are identical.
+constexpr int COMBINE_BATCH = 4;
+__device__ __forceinline__ void combine_small(const TileRec *tr, uint64_t replica_stride, uint32_t n_rep,
+                                              uint32_t nt, uint64_t nbytes, uint64_t k, uint32_t dtype,
+                                              uint64_t meta, uint64_t weight, uint32_t lane,
+                                              scout_sig_t (&o)[COMBINE_BATCH]) {
+    TileRec x[COMBINE_BATCH];
+#pragma unroll
+    for (int j = 0; j < COMBINE_BATCH; ++j) {
+        x[j].h = 0; x[j].sum = 0.0; x[j].sumsq = 0.0; x[j].nan_count = 0; x[j].inf_count = 0;
+        if ((uint32_t)j < n_rep && lane < nt) x[j] = load_record(tr + (uint64_t)j * replica_stride + lane);
+    }
+#pragma unroll
+    for (int j = 0; j < COMBINE_BATCH; ++j) {
+        uint64_t h = lane < nt - 1 ? x[j].h * weight : x[j].h;
+        double s = x[j].sum, q = x[j].sumsq;
+        uint32_t nan_count = x[j].nan_count, inf_count = x[j].inf_count;
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) {
+            h += __shfl_xor_sync(0xFFFFFFFFu, h, d);
+            s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
+            q += __shfl_xor_sync(0xFFFFFFFFu, q, d);
+            nan_count += __shfl_xor_sync(0xFFFFFFFFu, nan_count, d);
+            inf_count += __shfl_xor_sync(0xFFFFFFFFu, inf_count, d);
+        }
+        o[j].hash = finalize_hash(h, nbytes, k, dtype, meta);
+        o[j].nan_count = nan_count;
+        o[j].inf_count = inf_count;
+        o[j].sum = s;
+        o[j].sumsq = q;
+    }
+}
+
 
 __global__ void __launch_bounds__(FIN_THREADS) finalize_chunks(const ChunkDesc *chunks, uint64_t C,
                                                                uint32_t R, const TileRec *recs,
@@ -1065,13 +1129,323 @@ __global__ void __launch_bounds__(FIN_THREADS) finalize_chunks(const ChunkDesc *
         const uint32_t r = (uint32_t)(item - c * R);
         const ChunkDesc cd = chunks[c];
         const scout_sig_t o = combine_tiles(recs + (uint64_t)r * tiles_per_replica + cd.tile0, cd.ntiles,
-                                            cd.nbytes, cd.k, cd.dtype, cd.meta, tile_rows, p_stride, lane);
+                                            cd.nbytes, cd.k, cd.dtype, cd.meta, p_stride,
+                                            combine_weight(cd.ntiles, cd.nbytes, tile_rows, lane), lane);
         if (lane == 0) {
             sigs[c * R + r] = o;
         }
     }
 }
 
+
+// ---- one launch for the whole path --------------------------------------------------
+// certify_tiles = the direct scan + a per-chunk ticket.  Work items are taken tile-major
+// (item = tile * R + replica), so the chunks of the plan complete roughly in order.  The
+// warp that stores the last tile record of a chunk (atomic ticket; nobody waits for
+// anybody) finalises the chunk's R records and, in certify mode, votes the chunk, then
+// tries to advance the certificate chain: the chain is a strictly sequential fold over
+// the majority hashes in chunk order, so one warp at a time (a try-lock) folds whatever
+// prefix of chunks is complete and leaves; whoever completes the next chunk continues.
+// The warp that folds the last chunk writes the report block to pinned host memory and
+// returns the device state to zero for the next launch.  Nothing in the kernel spins.
+struct FusedArgs {
+    SignArgs s;
+    const ChunkDesc *chunks;
+    uint64_t C;
+    uint32_t R, tile_rows;
+    uint64_t p_stride;
+    scout_sig_t *sigs;
+    int mode;
+    VoteSinks v;
+    CertifyOut *out;
+    uint32_t *tickets;
+    uint32_t *done;
+    uint32_t epoch;
+    ChainState *chain;
+    CertifyHost *host;
+    unsigned long long *work;  // two work counters, used alternately by successive launches
+    uint32_t one_level;        // tickets: chunk counters only (chunks with few items)
+};
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_u32(uint32_t *p, uint32_t v) {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+constexpr uint64_t SMALL_CHAIN = 256;  // plans with at most this many chunks fold the chain in one go
+
+// The whole warp folds the complete prefix of chunks into the chain.  Returns true in
+// every lane if this warp folded the last chunk (it then still holds the lock and must
+// publish); chain_value is the finished chain in that case.
+__device__ __noinline__ bool advance_chain(const FusedArgs &a, uint32_t lane, uint64_t &chain_value) {
+    ChainState *ch = a.chain;
+    for (;;) {
+        uint32_t owner = 0;
+        if (lane == 0) owner = atomicCAS(&ch->lock, 0u, 1u) == 0u;
+        if (!__shfl_sync(0xFFFFFFFFu, owner, 0)) return false;  // another warp is folding; it re-checks after it
+        __threadfence();
+        uint64_t n = *(volatile uint64_t *)&ch->next;
+        uint64_t x = n ? *(volatile uint64_t *)&ch->a : mix64(SEED_CERT ^ a.C);
+        for (;;) {
+            const uint64_t c = n + lane;
+            uint64_t m = 0;
+            bool ready = false;
+            if (c < a.C && ld_acquire_u32(a.done + c) == a.epoch) {
+                ready = true;
+                m = __ldcg(a.v.majority + c);
+            }
+            const uint32_t mask = __ballot_sync(0xFFFFFFFFu, ready);
+            const uint32_t run = mask == 0xFFFFFFFFu ? 32u : (uint32_t)__ffs((int)~mask) - 1u;
+            for (uint32_t i = 0; i < run; ++i) x = mix64(x ^ __shfl_sync(0xFFFFFFFFu, m, i));
+            n += run;
+            if (run < 32u) break;
+        }
+        if (n == a.C) {
+            chain_value = x;
+            return true;
+        }
+        if (lane == 0) {
+            *(volatile uint64_t *)&ch->a = x;
+            *(volatile uint64_t *)&ch->next = n;
+            __threadfence();
+            atomicExch(&ch->lock, 0u);
+            __threadfence();
+        }
+        // a chunk may have completed between the last look and the release: look once more
+        uint32_t again = 0;
+        if (lane == 0) again = ld_acquire_u32(a.done + n) == a.epoch;
+        if (!__shfl_sync(0xFFFFFFFFu, again, 0)) return false;
+    }
+}
+
+// Every chunk has been voted and folded: finish the counters, write the report block to
+// the host and leave the device state zero.  Called by one warp, which holds the chain lock.
+__device__ __noinline__ void publish_report(const FusedArgs &a, uint32_t lane, uint64_t chain_value) {
+    uint64_t *dev = reinterpret_cast<uint64_t *>(a.out);
+    volatile uint64_t *host = reinterpret_cast<volatile uint64_t *>(&a.host->out);
+    constexpr uint32_t WORDS = sizeof(CertifyOut) / sizeof(uint64_t);
+    const uint64_t n_inconclusive = __ldcg(&a.out->counts[3]);
+    const uint64_t n_out = __ldcg(&a.out->counts[4]), n_und = __ldcg(&a.out->counts[5]);
+    for (uint32_t i = lane; i < WORDS; i += 32) {
+        uint64_t w = __ldcg(dev + i);
+        if (i == 0) w = a.C;                                           // counts[0]
+        if (i == 7) w = n_inconclusive ? 0ull : chain_value;           // certificate
+        host[i] = w;
+        dev[i] = 0ull;                                                 // zero for the next launch
+    }
+    static_assert(offsetof(CertifyOut, certificate) == 7 * sizeof(uint64_t), "word 7 is the certificate");
+    const uint64_t head_out = min(min(n_out, a.v.outlier_cap), CERTIFY_HEAD);
+    const uint64_t head_und = min(min(n_und, a.v.undecided_cap), CERTIFY_HEAD);
+    for (uint64_t i = lane; i < 2 * head_out; i += 32)
+        reinterpret_cast<volatile uint64_t *>(a.host->outliers)[i] =
+            __ldcg(reinterpret_cast<const uint64_t *>(a.v.outliers) + i);
+    for (uint64_t i = lane; i < head_und; i += 32)
+        reinterpret_cast<volatile uint64_t *>(a.host->undecided)[i] = __ldcg(a.v.undecided + i);
+    if (lane == 0) {
+        *reinterpret_cast<volatile uint32_t *>(&a.host->dev_err) = a.s.error ? __ldcg(a.s.error) : 0u;
+        *(volatile uint64_t *)&a.chain->next = 0ull;
+        *(volatile uint64_t *)&a.chain->a = 0ull;
+        __threadfence_system();
+        atomicExch(&a.chain->lock, 0u);
+    }
+}
+
+// The last tile record of chunk c has been stored: finalise, vote, fold.
+__device__ __noinline__ void chunk_complete(const FusedArgs &a, uint32_t c, uint32_t lane) {
+    __threadfence();  // the records the other warps released before their tickets are visible now
+    const ChunkDesc cd = a.chunks[c];
+    uint64_t e0 = 0, e1 = 0;
+    const uint64_t weight = combine_weight(cd.ntiles, cd.nbytes, a.tile_rows, lane);
+    const TileRec *tr = a.s.recs + cd.tile0;
+    if (cd.ntiles <= 32u) {
+        for (uint32_t r0 = 0; r0 < a.R; r0 += COMBINE_BATCH) {
+            scout_sig_t o[COMBINE_BATCH];
+            const uint32_t n_rep = min((uint32_t)COMBINE_BATCH, a.R - r0);
+            combine_small(tr + (uint64_t)r0 * a.s.tiles_per_replica, a.s.tiles_per_replica, n_rep, cd.ntiles,
+                          cd.nbytes, cd.k, cd.dtype, cd.meta, weight, lane, o);
+#pragma unroll
+            for (int j = 0; j < COMBINE_BATCH; ++j) {
+                const uint32_t r = r0 + j;
+                if (r < a.R) {
+                    if (lane == 0) a.sigs[(uint64_t)c * a.R + r] = o[j];
+                    if (lane == (r & 31u)) {
+                        if (r < 32u) e0 = o[j].hash; else e1 = o[j].hash;
+                    }
+                }
+            }
+        }
+    } else {
+        for (uint32_t r = 0; r < a.R; ++r) {
+            const scout_sig_t o = combine_tiles(tr + (uint64_t)r * a.s.tiles_per_replica, cd.ntiles, cd.nbytes,
+                                                cd.k, cd.dtype, cd.meta, a.p_stride, weight, lane);
+            if (lane == 0) a.sigs[(uint64_t)c * a.R + r] = o;
+            const uint64_t h = __shfl_sync(0xFFFFFFFFu, o.hash, 0);
+            if (lane == (r & 31u)) {
+                if (r < 32u) e0 = h; else e1 = h;
+            }
+        }
+    }
+    // both ticket levels of this chunk go back to zero for the next launch
+    for (uint32_t r = lane; r <= a.R; r += 32) a.tickets[r < a.R ? (uint64_t)c * a.R + r : a.C * a.R + c] = 0u;
+    if (a.mode == 0) return;
+    uint64_t bitmap, majority;
+    const uint32_t st = vote_chunk(a.R, c, e0, e1, lane, a.v, bitmap, majority);
+    if (a.C <= SMALL_CHAIN) {
+        // Few chunks: no incremental folding.  The warp that votes the last chunk folds the
+        // whole chain at once (C mix steps after one round of loads).
+        uint32_t finisher = 0;
+        if (lane == 0) {
+            atomicAdd((unsigned long long *)&a.out->counts[1 + st], 1ull);  // AGREE, ATTRIBUTED, INCONCLUSIVE
+            if (bitmap) atomicOr((unsigned long long *)&a.out->union_bitmap, (unsigned long long)bitmap);
+            __threadfence();
+            finisher = atomicAdd((unsigned long long *)&a.chain->next, 1ull) + 1ull == a.C;
+        }
+        if (!__shfl_sync(0xFFFFFFFFu, finisher, 0)) return;
+        __threadfence();
+        uint64_t x = mix64(SEED_CERT ^ a.C);
+        for (uint64_t base = 0; base < a.C; base += 32) {
+            const uint64_t m = base + lane < a.C ? __ldcg(a.v.majority + base + lane) : 0ull;
+            const uint32_t n = (uint32_t)min((uint64_t)32, a.C - base);
+            for (uint32_t i = 0; i < n; ++i) x = mix64(x ^ __shfl_sync(0xFFFFFFFFu, m, i));
+        }
+        publish_report(a, lane, x);
+        return;
+    }
+    if (lane == 0) {
+        atomicAdd((unsigned long long *)&a.out->counts[1 + st], 1ull);
+        if (bitmap) atomicOr((unsigned long long *)&a.out->union_bitmap, (unsigned long long)bitmap);
+        __threadfence();
+        st_release_u32(a.done + c, a.epoch);
+        __threadfence();
+    }
+    __syncwarp();
+    uint64_t chain_value = 0;
+    if (advance_chain(a, lane, chain_value)) publish_report(a, lane, chain_value);
+}
+
+// Tickets.  First level: one counter per (chunk, replica), advanced once per tile; the warp
+// that brings it to the chunk's tile count advances the second level, one counter per
+// chunk, and the warp that brings that one to R has completed the chunk.  Two levels keep
+// the number of atomics per address small (same-address atomics serialise in L2); plans
+// whose chunks have few (tile, replica) items use the chunk counter alone (one round trip
+// less on the way to the result).  The result of a tile's atomic is looked at one tile
+// later, after the next tile has been scanned, so no warp waits for an atomic's round trip.
+__device__ __forceinline__ void resolve_ticket(const FusedArgs &a, uint32_t lane, uint32_t returned,
+                                               uint32_t tiles_of_chunk, uint32_t chunk) {
+    uint32_t last = 0;
+    if (a.one_level) {
+        last = lane == 0 && returned + 1u == tiles_of_chunk * a.R;
+    } else if (lane == 0 && returned + 1u == tiles_of_chunk) {
+        last = atomicAdd(&a.tickets[a.C * a.R + chunk], 1u) + 1u == a.R;
+    }
+    if (__shfl_sync(0xFFFFFFFFu, last, 0)) chunk_complete(a, chunk, lane);
+}
+
+template <int DTSEL>
+__global__ void __launch_bounds__(SIGN_THREADS, SCOUT_MINBLOCKS) certify_tiles(const __grid_constant__ FusedArgs a) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint64_t warp = (uint64_t)blockIdx.x * (SIGN_THREADS / 32) + (threadIdx.x >> 5);
+    const uint64_t n_warps = (uint64_t)gridDim.x * (SIGN_THREADS / 32);
+    const uint64_t n_items = a.s.n_tiles * a.R;
+    // Work items are handed out dynamically (a warp that stops to finalise a chunk simply
+    // takes fewer tiles afterwards): every warp starts with item `warp`, later items come
+    // from a counter.  The counter of this launch is work[epoch & 1]; the other one is
+    // zeroed here for the next launch.  The next item is requested before the current tile
+    // is scanned and looked at after it, so the atomic's round trip is never waited for.
+    unsigned long long *work = a.work + (a.epoch & 1u);
+    if (warp == 0 && lane == 0) a.work[(a.epoch & 1u) ^ 1u] = 0ull;
+    // the previous tile's ticket: value its atomic returned (lane 0), tiles of its chunk, its chunk
+    uint32_t prev_returned = 0, prev_tiles = 0, prev_chunk = 0;
+    const bool more_rounds = n_items > n_warps;  // otherwise every warp has at most its first item
+    uint64_t item = warp;
+    while (item < n_items) {
+        unsigned long long next = n_items;  // "nothing left" unless the counter says otherwise
+        if (more_rounds && lane == 0) next = atomicAdd(work, 1ull);
+        const uint64_t t = item / a.R;
+        const uint32_t r = (uint32_t)(item - t * a.R);
+        const TileDesc td = a.s.tiles[t];
+        const uint8_t *tile = a.s.ptrs[(uint64_t)r * a.s.T + td.tensor] + td.off;
+        // whoever completes this chunk reads its descriptor: have it in L2 by then
+        if (lane == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(a.chunks + td.chunk));
+        TileRec rec;
+        if constexpr (DTSEL >= 0) scan_tile<DTSEL>(tile, td.nbytes, lane, rec);
+        else                      scan_dispatch(td.dtype, tile, td.nbytes, lane, rec);
+        if (prev_tiles) resolve_ticket(a, lane, prev_returned, prev_tiles, prev_chunk);
+        if (lane == 0) {
+            store_record(&a.s.recs[(uint64_t)r * a.s.tiles_per_replica + t], rec);
+            __threadfence();
+            prev_returned = atomicAdd(&a.tickets[a.one_level ? a.C * a.R + td.chunk : (uint64_t)td.chunk * a.R + r], 1u);
+        }
+        prev_tiles = td.chunk_tiles;
+        prev_chunk = td.chunk;
+        item = n_warps + __shfl_sync(0xFFFFFFFFu, next, 0);
+    }
+    if (prev_tiles) resolve_ticket(a, lane, prev_returned, prev_tiles, prev_chunk);
+}
+
+using FusedKernel = void (*)(const FusedArgs);
+FusedKernel fused_kernel(int uniform) {
+    if (uniform == SCOUT_DT_F32) return certify_tiles<SCOUT_DT_F32>;
+    if (uniform == SCOUT_DT_BF16) return certify_tiles<SCOUT_DT_BF16>;
+    return certify_tiles<-1>;
+}
+
+}  // namespace
+
+int fused_grid_size(int uniform_dtype, int device, int *grid) {
+    int sms = 0, per_sm = 0;
+    SCOUT_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+    SCOUT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_kernel(uniform_dtype), SIGN_THREADS, 0));
+    if (per_sm < 1) per_sm = 1;
+    *grid = sms * per_sm;
+    return SCOUT_OK;
+}
+
+int launch_fused(const FusedLaunch &l, cudaStream_t stream) {
+    if (l.sign.n_tiles == 0 || l.R == 0) return SCOUT_OK;
+    FusedArgs a;
+    a.s.tiles = l.sign.tiles;
+    a.s.tile_begin = 0;
+    a.s.n_tiles = l.sign.n_tiles;
+    a.s.tiles_per_replica = l.sign.tiles_per_replica;
+    a.s.replica_begin = 0;
+    a.s.n_replicas = l.R;
+    a.s.ptrs = l.sign.ptrs;
+    a.s.T = l.sign.T;
+    a.s.stage = nullptr;
+    a.s.slice_begin = 0;
+    a.s.recs = l.sign.recs;
+    a.s.error = l.sign.error;
+    a.chunks = l.chunks;
+    a.C = l.C;
+    a.R = l.R;
+    a.tile_rows = l.tile_rows;
+    a.p_stride = pow_p(32ull * l.tile_rows);
+    a.sigs = l.sigs;
+    a.mode = l.mode;
+    a.v = l.vote;
+    a.out = l.out;
+    a.tickets = l.tickets;
+    a.done = l.done;
+    a.epoch = l.epoch;
+    a.chain = l.chain;
+    a.host = l.host;
+    a.work = l.work;
+    a.one_level = l.one_level;
+    const uint64_t items = l.sign.n_tiles * l.R;
+    const uint64_t want = (items + SIGN_THREADS / 32 - 1) / (SIGN_THREADS / 32);
+    int grid = l.sign.grid;
+    if ((uint64_t)grid > want) grid = (int)want;
+    fused_kernel(l.sign.uniform_dtype)<<<grid, SIGN_THREADS, 0, stream>>>(a);
+    SCOUT_CUDA(cudaGetLastError());
+    return SCOUT_OK;
+}
+
+namespace {
 }  // namespace
 
 int sign_grid_size(int variant, int uniform_dtype, int device, int *grid) {
@@ -1214,7 +1588,8 @@ __global__ void __launch_bounds__(FIN_THREADS) finalize_noalloc(const __grid_con
         const uint64_t chunk_n = min(a.chunk_bytes, a.nbytes - c * a.chunk_bytes);
         const uint32_t nt = (uint32_t)((chunk_n + a.tile_bytes - 1) / a.tile_bytes);
         const scout_sig_t o = combine_tiles(a.recs + (uint64_t)r * a.n_tiles + c * a.tiles_per_chunk, nt,
-                                            chunk_n, c, a.dtype, a.meta, tile_rows, p_stride, lane);
+                                            chunk_n, c, a.dtype, a.meta, p_stride,
+                                            combine_weight(nt, chunk_n, tile_rows, lane), lane);
         if (lane == 0) {
             a.sigs[c * a.R + r] = o;
         }

@@ -2,16 +2,14 @@
 // evidence of every chunk, the compaction of disagreements into lists, and the
 // roll-ups built on top of it.
 #include "scout_internal.h"
+#include "scout_vote_device.cuh"
 
 namespace scout {
 namespace {
 
 constexpr int VOTE_THREADS = 256;
 
-// One warp per chunk.  Lane j holds e_j and e_{j+32}.  cnt_j = #{i : e_i = e_j};
-// c* = max cnt.  2 c* <= R: Inconclusive, bitmap 0.  Otherwise e* is the unique
-// value with count c*, bit j = 1{e_j != e*}.  Outlier pairs and undecided chunk
-// ids are appended with one atomic per warp.
+// One warp per chunk; the rule itself is vote_chunk() (scout_vote_device.cuh).
 __global__ void __launch_bounds__(VOTE_THREADS) vote_chunks(
     uint32_t R, uint64_t C, const scout_sig_t *__restrict__ sigs, uint8_t *status_out,
     uint64_t *bitmap_out, scout_outlier_t *outliers, uint64_t outlier_cap, uint64_t *undecided,
@@ -23,76 +21,19 @@ __global__ void __launch_bounds__(VOTE_THREADS) vote_chunks(
     const uint64_t n_warps = (uint64_t)gridDim.x * (VOTE_THREADS / 32);
     uint32_t n_agree = 0, n_attr = 0, n_inc = 0;  // per warp, identical in all lanes
     uint64_t union_bits = 0;
+    const VoteSinks sinks = {status_out, bitmap_out, majority_out, outliers, outlier_cap,
+                             undecided, undecided_cap, counts, cert};
 
     for (uint64_t c = warp; c < C; c += n_warps) {
         const scout_sig_t *e = sigs + c * R;
-        const bool have0 = lane < R, have1 = lane + 32u < R;
-        const uint64_t e0 = have0 ? e[lane].hash : 0ull;
-        const uint64_t e1 = have1 ? e[lane + 32u].hash : 0ull;
-        uint32_t cnt0 = 0, cnt1 = 0;
-        for (uint32_t i = 0; i < R; ++i) {
-            const uint64_t lo = __shfl_sync(0xFFFFFFFFu, e0, i & 31u);
-            const uint64_t hi = __shfl_sync(0xFFFFFFFFu, e1, i & 31u);
-            const uint64_t ei = i < 32u ? lo : hi;
-            cnt0 += (ei == e0);
-            cnt1 += (ei == e1);
-        }
-        if (!have0) cnt0 = 0;
-        if (!have1) cnt1 = 0;
-        const uint32_t mine = cnt0 > cnt1 ? cnt0 : cnt1;
-        const uint32_t best = __reduce_max_sync(0xFFFFFFFFu, mine);
-
-        uint64_t bitmap = 0, majority = 0;
-        uint32_t st;
-        if (2u * best <= R) {
-            st = SCOUT_INCONCLUSIVE;
-            ++n_inc;
-        } else {
-            // the lanes holding e* (count == best) agree on one value
-            const uint32_t holders = __ballot_sync(0xFFFFFFFFu, cnt0 == best);
-            const uint32_t holders_hi = __ballot_sync(0xFFFFFFFFu, cnt1 == best);
-            if (holders) majority = __shfl_sync(0xFFFFFFFFu, e0, __ffs(holders) - 1);
-            else         majority = __shfl_sync(0xFFFFFFFFu, e1, __ffs(holders_hi) - 1);
-            const uint32_t b0 = __ballot_sync(0xFFFFFFFFu, have0 && e0 != majority);
-            const uint32_t b1 = __ballot_sync(0xFFFFFFFFu, have1 && e1 != majority);
-            bitmap = ((uint64_t)b1 << 32) | b0;
-            st = bitmap ? SCOUT_ATTRIBUTED : SCOUT_AGREE;
-            if (bitmap) ++n_attr; else ++n_agree;
-            union_bits |= bitmap;
-        }
-        if (lane == 0) {
-            if (status_out) status_out[c] = (uint8_t)st;
-            if (bitmap_out) bitmap_out[c] = bitmap;
-            if (majority_out) majority_out[c] = majority;
-        }
-        if (bitmap) {  // warp-aggregated append of (chunk, replica) pairs
-            const uint32_t n = __popcll(bitmap);
-            unsigned long long base = 0;
-            if (lane == 0) base = atomicAdd((unsigned long long *)&counts[4], (unsigned long long)n);
-            base = __shfl_sync(0xFFFFFFFFu, base, 0);
-            const uint32_t b0 = (uint32_t)bitmap, b1 = (uint32_t)(bitmap >> 32);
-            const uint32_t below = (1u << lane) - 1u;
-            if ((b0 >> lane) & 1u) {
-                const uint64_t pos = base + __popc(b0 & below);
-                if (pos < outlier_cap) outliers[pos] = scout_outlier_t{c, lane, 0u};
-            }
-            if ((b1 >> lane) & 1u) {
-                const uint64_t pos = base + __popc(b0) + __popc(b1 & below);
-                if (pos < outlier_cap) outliers[pos] = scout_outlier_t{c, lane + 32u, 0u};
-            }
-            if (cert && lane == 0) {
-                uint64_t b = bitmap;
-                while (b) {
-                    const int j = __ffsll((long long)b) - 1;
-                    atomicAdd((unsigned long long *)&cert->replica_bad[j], 1ull);
-                    b &= b - 1;
-                }
-            }
-        }
-        if (st == SCOUT_INCONCLUSIVE && lane == 0) {
-            const unsigned long long pos = atomicAdd((unsigned long long *)&counts[5], 1ull);
-            if (pos < undecided_cap) undecided[pos] = c;
-        }
+        const uint64_t e0 = lane < R ? e[lane].hash : 0ull;
+        const uint64_t e1 = lane + 32u < R ? e[lane + 32u].hash : 0ull;
+        uint64_t bitmap, majority;
+        const uint32_t st = vote_chunk(R, c, e0, e1, lane, sinks, bitmap, majority);
+        if (st == SCOUT_INCONCLUSIVE) ++n_inc;
+        else if (st == SCOUT_ATTRIBUTED) ++n_attr;
+        else ++n_agree;
+        union_bits |= bitmap;
     }
 
     // block-level aggregation of the status counters: one atomic per counter per CTA

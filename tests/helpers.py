@@ -68,7 +68,11 @@ def gpu_plan(w, chunk_bytes=None, tags=None, tile_bytes=None, variant=None):
                         w.chunk_bytes if chunk_bytes is None else chunk_bytes)
     if tile_bytes is not None:
         binding.scout_plan_set(plan.handle, "tile_bytes", tile_bytes)
-    if variant is not None:
+    if variant == "unfused":      # the default scan, one kernel per stage
+        binding.scout_plan_set(plan.handle, "fused", 0)
+    elif variant == "fused":      # the default scan, the whole call as one launch
+        binding.scout_plan_set(plan.handle, "fused", 1)
+    elif variant is not None:
         binding.scout_plan_set(plan.handle, "variant", variant)
     return plan
 
