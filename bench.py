@@ -66,6 +66,7 @@ def parse_args():
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--variant", type=int, default=None)
     ap.add_argument("--tile-bytes", type=int, default=None)
+    ap.add_argument("--fused", type=int, default=None, help="plan key 'fused': 1, 0 or -1 (default)")
     ap.add_argument("--also", default=None,
                     help="comma-separated configs measured after the headline one and reported under "
                          "'also' (default: 3,5 for the default full-size run at N=1; '' for none)")
@@ -273,6 +274,8 @@ def run_config(cfg, args, rank, world, local, headline):
         binding.scout_plan_set(plan.handle, "tile_bytes", args.tile_bytes)
     if args.variant is not None:
         binding.scout_plan_set(plan.handle, "variant", args.variant)
+    if args.fused is not None:
+        binding.scout_plan_set(plan.handle, "fused", args.fused)
     plan.bind(views)
     use_certify = cfg == 4
 

@@ -279,9 +279,11 @@ SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/)
  *                     last chunk writes the report block to pinned host memory.
  *                     1: always; 0: never (one kernel per stage: scan, finalise, vote,
  *                     certificate - the form scout_certify_host always uses); -1
- *                     (default): where it is the faster form - scout_certify always;
- *                     scout_sign_chunks for plans of 1 GB and more whose tensors are all
- *                     fp32 or all bf16
+ *                     (default): where it measured faster - scout_certify on plans below
+ *                     1 GB (latency: one launch instead of four and the copies); larger
+ *                     plans and scout_sign_chunks run the stages as separate kernels
+ *   set "dynamic"     1 (default): the scan's warps take tiles from a work counter as they
+ *                     become free; 0: fixed round-robin assignment
  *   set "grid"        CTAs of the scan kernel
  *   set "timing"      1: record a pair of CUDA events around every scan kernel on
  *                     the caller's stream (a ring of 256 pairs); setting it again

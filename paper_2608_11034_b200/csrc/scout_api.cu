@@ -73,7 +73,10 @@ struct scout_plan {
     int fused_grid = 0;
     uint32_t *d_tickets = nullptr, *d_done = nullptr;
     ChainState *d_chain = nullptr;
-    unsigned long long *d_work = nullptr;
+    unsigned long long *d_work = nullptr;   // one-launch kernels
+    unsigned long long *d_work2 = nullptr;  // direct scan kernels of the staged path
+    uint64_t work_launches = 0;
+    bool dynamic = true;                    // key "dynamic"
     CertifyHost *h_out_dev = nullptr;  // device-side address of h_out
     uint32_t epoch = 0;
     bool out_dirty = false;       // d_out was left non-zero by the multi-kernel path
@@ -161,20 +164,20 @@ int upload_tables(scout_plan *p) {
     return SCOUT_OK;
 }
 
-// Is this call made as one launch?  Measured on B200.  scout_certify: always - one kernel
-// instead of four plus the copies is faster at every size (12.6 MB: 34 against 42 us on the
-// device, 51 against 67 us per call; 36 GB: +1 %), and from a few thousand chunks on it also
-// hides the sequential certificate chain behind the scan.  scout_sign_chunks alone: only for
-// plans of 1 GB and more whose tensors are all fp32 or all bf16.  Below that the scan and the
-// finalise kernel launched back to back (programmatic dependent launch) are faster, because the
-// ticket and the finalisation by the last warp add L2 round trips of about a microsecond each
-// to a kernel that runs for tens of microseconds; and the kernel that reads the dtype from the
-// tile table spills registers in its one-launch form (-2 % on 10,000 mixed tensors).
+// Is this call made as one launch?  Measured on B200 (key "fused" = -1, the default, follows
+// the measurements; 1 and 0 force either form):
+//   * scout_certify on plans below 1 GB: yes.  One kernel instead of four plus the copies
+//     (12.6 MB: 34 against 42 us on the device, 51 against 67 us per call).
+//   * everything else: no.  With its work handed out dynamically the staged scan reaches
+//     7.2 TB/s on 36 GB of fp32 and 6.25 TB/s on 125 GB of bf16; the one-launch kernel, whose
+//     loop also carries the ticket state (it spills) and takes tiles replica-interleaved, stays
+//     3 to 7 % below that, more than the three small launches it saves.  What the one-launch
+//     form alone offers at large sizes is the certificate chain folded behind the scan (39 ns
+//     per chunk otherwise: 28 us at 717 chunks, 0.9 ms at 24,000).
 bool use_fused(const scout_plan *p, bool certify) {
     if (p->variant != 0 || p->R > 64 || !p->d_tickets || p->fused == 0) return false;
-    if (p->fused > 0 || certify) return true;
-    return p->total_bytes >= (1ull << 30) &&
-           (p->uniform_dtype == SCOUT_DT_F32 || p->uniform_dtype == SCOUT_DT_BF16);
+    if (p->fused > 0) return true;
+    return certify && p->total_bytes < (1ull << 30);
 }
 
 void fill_sign_launch(const scout_plan *p, SignLaunch &l) {
@@ -193,6 +196,15 @@ void fill_sign_launch(const scout_plan *p, SignLaunch &l) {
     l.variant = p->variant;
     l.uniform_dtype = p->uniform_dtype;
     l.grid = p->grid;
+    l.work = nullptr;
+    l.work_parity = 0;
+}
+
+// The direct scan kernels take their work dynamically: successive launches alternate between
+// the plan's two counters (the launch that uses one zeroes the other).
+void next_work_counter(scout_plan *p, SignLaunch &l) {
+    l.work = p->dynamic ? p->d_work2 : nullptr;
+    l.work_parity = (p->work_launches++) & 1u;
 }
 
 // One kernel: scan + finalise (certify == false), or the whole certify path.  The timing
@@ -242,21 +254,8 @@ int launch_one_kernel(scout_plan *p, cudaStream_t stream, scout_sig_t *d_sigs, b
 int sign_all(scout_plan *p, cudaStream_t stream, scout_sig_t *d_sigs, CertifyOut *zero_out = nullptr) {
     if (use_fused(p, false) && !zero_out) return launch_one_kernel(p, stream, d_sigs, false, 0, 0);
     SignLaunch l;
-    l.tiles = p->d_tiles;
-    l.tile_begin = 0;
-    l.n_tiles = p->tiles.size();
-    l.tiles_per_replica = p->tiles.size();
-    l.replica_begin = 0;
-    l.n_replicas = p->R;
-    l.ptrs = (const uint8_t *const *)p->d_ptrs;
-    l.T = p->T;
-    l.stage = nullptr;
-    l.slice_begin = 0;
-    l.recs = p->d_recs;
-    l.error = p->d_error;
-    l.variant = p->variant;
-    l.uniform_dtype = p->uniform_dtype;
-    l.grid = p->grid;
+    fill_sign_launch(p, l);
+    next_work_counter(p, l);
     const size_t slot = p->timing ? (size_t)(p->timed_launches % p->ev_t0.size()) : 0;
     if (p->timing) SCOUT_CUDA(cudaEventRecord(p->ev_t0[slot], stream));
     int rc = launch_sign_tiles(l, stream);
@@ -480,14 +479,16 @@ int scout_plan_create(uint32_t R, uint64_t T, const scout_tensor_t *tensors, uin
         if (cudaMalloc(&p->d_tickets, n_tickets * sizeof(uint32_t)) != cudaSuccess ||
             cudaMalloc(&p->d_done, nc * sizeof(uint32_t)) != cudaSuccess ||
             cudaMalloc(&p->d_chain, sizeof(ChainState)) != cudaSuccess ||
-            cudaMalloc(&p->d_work, 2 * sizeof(unsigned long long)) != cudaSuccess) {
+            cudaMalloc(&p->d_work, 2 * sizeof(unsigned long long)) != cudaSuccess ||
+            cudaMalloc(&p->d_work2, 2 * sizeof(unsigned long long)) != cudaSuccess) {
             rc = SCOUT_ERR_NOMEM;
             break;
         }
         if (cudaMemset(p->d_tickets, 0, n_tickets * sizeof(uint32_t)) != cudaSuccess ||
             cudaMemset(p->d_done, 0, nc * sizeof(uint32_t)) != cudaSuccess ||
             cudaMemset(p->d_chain, 0, sizeof(ChainState)) != cudaSuccess ||
-            cudaMemset(p->d_work, 0, 2 * sizeof(unsigned long long)) != cudaSuccess) {
+            cudaMemset(p->d_work, 0, 2 * sizeof(unsigned long long)) != cudaSuccess ||
+            cudaMemset(p->d_work2, 0, 2 * sizeof(unsigned long long)) != cudaSuccess) {
             rc = SCOUT_ERR_CUDA;
             break;
         }
@@ -556,6 +557,7 @@ int scout_plan_destroy(scout_plan_t *p) {
     cudaFree(p->d_done);
     cudaFree(p->d_chain);
     cudaFree(p->d_work);
+    cudaFree(p->d_work2);
     cudaFree(p->d_sigs);
     cudaFree(p->d_status);
     cudaFree(p->d_bitmap);
@@ -725,6 +727,7 @@ int scout_certify_host(scout_plan_t *p, const void *const *h_ptrs, scout_report_
             l.variant = p->variant == 3 ? 0 : p->variant;
             l.uniform_dtype = p->uniform_dtype;
             l.grid = p->grid;
+            next_work_counter(p, l);
             if ((rc = launch_sign_tiles(l, p->s_comp))) return rc;
             SCOUT_CUDA(cudaEventRecord(p->ev_done[buf], p->s_comp));
             t0 = t1;
@@ -802,6 +805,10 @@ int scout_plan_set(scout_plan_t *p, const char *key, int64_t value) {
         }
         return upload_tables(p);
     }
+    if (!std::strcmp(key, "dynamic")) {
+        p->dynamic = value != 0;
+        return SCOUT_OK;
+    }
     if (!std::strcmp(key, "fused")) {
         if (value < -1 || value > 1) return SCOUT_ERR_INVALID;
         p->fused = (int)value;
@@ -845,6 +852,7 @@ int scout_plan_get(const scout_plan_t *p, const char *key, int64_t *value) {
     else if (!std::strcmp(key, "grid")) *value = p->grid;
     else if (!std::strcmp(key, "n_tiles")) *value = (int64_t)p->tiles.size();
     else if (!std::strcmp(key, "fused")) *value = p->fused;
+    else if (!std::strcmp(key, "dynamic")) *value = p->dynamic;
     else if (!std::strcmp(key, "sign_kernels")) *value = use_fused(p, false) ? 1 : 2;    // scan, finalise
     else if (!std::strcmp(key, "certify_kernels")) *value = use_fused(p, true) ? 1 : 4;  // + vote, certificate chain
     else if (!std::strcmp(key, "last_sign_ns")) {

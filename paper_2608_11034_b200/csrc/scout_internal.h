@@ -182,6 +182,8 @@ struct SignLaunch {
     uint32_t *error;              // device flag set when a bounded wait gave up (may be null)
     int variant;                  // 0 direct, 1 direct + register prefetch, 2 bulk-async ring, 3 read probe
     int uniform_dtype;            // dtype shared by every tile of the launch, or -1 if they differ
+    unsigned long long *work;     // device [2] work counters of the direct scan (null: fixed round-robin)
+    uint32_t work_parity;         // which of the two this launch uses (successive launches alternate)
     int grid;                     // CTAs to launch
 };
 int launch_sign_tiles(const SignLaunch &a, cudaStream_t stream);

@@ -397,6 +397,10 @@ struct SignArgs {
     uint64_t slice_begin;
     TileRec *recs;
     uint32_t *error;  // device flag: set if a bounded wait gave up
+    // dynamic work distribution of the direct scan: two counters used alternately by
+    // successive launches (null: static round-robin), and this launch's parity
+    unsigned long long *work;
+    uint32_t work_parity;
 };
 
 __device__ __forceinline__ void scan_dispatch(uint32_t dtype, const uint8_t *tile, uint32_t nbytes,
@@ -448,7 +452,20 @@ __global__ void __launch_bounds__(SIGN_THREADS, PREFETCH ? SCOUT_MINBLOCKS_PF : 
     const uint64_t warp = (uint64_t)blockIdx.x * (SIGN_THREADS / 32) + (threadIdx.x >> 5);
     const uint64_t n_warps = (uint64_t)gridDim.x * (SIGN_THREADS / 32);
     const uint64_t n_items = a.n_tiles * a.n_replicas;
-    for (uint64_t item = warp; item < n_items; item += n_warps) {
+    // Every warp starts with item `warp`.  With a work counter the later items are handed out
+    // in order as warps become free (tiles differ in size and dtype, so a fixed round-robin
+    // leaves some warps with more bytes than others); the request for the next item is made
+    // before the current tile is scanned and its answer is read after it.  The counter of this
+    // launch is work[parity]; the other one is zeroed here for the launch that follows.
+    unsigned long long *work = a.work ? a.work + a.work_parity : nullptr;
+    if (work && warp == 0 && lane == 0) a.work[a.work_parity ^ 1u] = 0ull;
+    const bool dynamic = work != nullptr && n_items > n_warps;
+    uint64_t item = warp;
+    while (item < n_items) {
+        unsigned long long next = 0;
+        if (dynamic) {
+            if (lane == 0) next = atomicAdd(work, 1ull);
+        }
         const uint32_t rr = (uint32_t)(item / a.n_tiles);
         const uint64_t t = a.tile_begin + (item - (uint64_t)rr * a.n_tiles);
         const uint32_t r = a.replica_begin + rr;
@@ -463,6 +480,7 @@ __global__ void __launch_bounds__(SIGN_THREADS, PREFETCH ? SCOUT_MINBLOCKS_PF : 
             else          scan_dispatch(td.dtype, tile, td.nbytes, lane, rec);
         }
         if (lane == 0) store_record(&a.recs[(uint64_t)r * a.tiles_per_replica + t], rec);
+        item = dynamic ? n_warps + __shfl_sync(0xFFFFFFFFu, next, 0) : item + n_warps;
     }
 }
 
@@ -1420,6 +1438,8 @@ int launch_fused(const FusedLaunch &l, cudaStream_t stream) {
     a.s.slice_begin = 0;
     a.s.recs = l.sign.recs;
     a.s.error = l.sign.error;
+    a.s.work = nullptr;
+    a.s.work_parity = 0;
     a.chunks = l.chunks;
     a.C = l.C;
     a.R = l.R;
@@ -1481,6 +1501,8 @@ int launch_sign_tiles(const SignLaunch &l, cudaStream_t stream) {
     a.slice_begin = l.slice_begin;
     a.recs = l.recs;
     a.error = l.error;
+    a.work = l.work;
+    a.work_parity = l.work_parity;
     const uint64_t items = l.n_tiles * l.n_replicas;
     const uint64_t want = (items + SIGN_THREADS / 32 - 1) / (SIGN_THREADS / 32);
     int grid = l.grid;
