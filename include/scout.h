@@ -263,7 +263,7 @@ SCOUT_API int scout_sign_chunks_noalloc(uint32_t R, const void *const *replica_p
 SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/);
 
 /* Knobs of a plan (optional).
- *   set "tile_bytes"  bytes per work item, a power of two in [2048, 65536]
+ *   set "tile_bytes"  bytes per work item, a power of two in [2048, 262144]
  *   set "variant"     scan kernel: 0 = direct 16-byte loads (default); 1 = the same
  *                     with the next rows prefetched into registers; 2 = bulk-async
  *                     copies (cp.async.bulk + mbarrier) through a per-warp ring in

@@ -50,9 +50,12 @@ constexpr int SIGN_THREADS = 256;
 
 constexpr int UNROLL = SCOUT_UNROLL;
 // bf16: how many of a word-quad's four high halves are widened by bit placement
-// instead of the conversion pipe (see stats_fast).
+// instead of the conversion pipe (see stats_fast).  Default 0: every instruction costs about
+// 1.6 issue cycles whatever its pipe, so the route with the fewest instructions wins even
+// though it keeps the conversion pipe busiest (measured on 125 GB of bf16: 6,361 GB/s with 0,
+// 6,282 with 1, 6,223 with 2, 6,016 with 3).
 #ifndef SCOUT_BF16_BITROUTE
-#define SCOUT_BF16_BITROUTE 2
+#define SCOUT_BF16_BITROUTE 0
 #endif
 
 constexpr int BF16_BITROUTE = SCOUT_BF16_BITROUTE;

@@ -23,7 +23,7 @@ def test_plan_knobs():
     B.scout_plan_set(h, "tile_bytes", 2048)
     assert B.scout_plan_get(h, "n_tiles") == w.bytes_per_replica // 2048 != n0
     assert B.scout_plan_get(h, "scratch_bytes") == B.scout_plan_get(h, "n_tiles") * w.R * 32
-    for key, bad in (("tile_bytes", 1000), ("tile_bytes", 131072), ("variant", 5), ("variant", -1),
+    for key, bad in (("tile_bytes", 1000), ("tile_bytes", 524288), ("variant", 5), ("variant", -1),
                      ("grid", 0), ("nonsense", 1)):
         with pytest.raises(B.ScoutError):
             B.scout_plan_set(h, key, bad)
