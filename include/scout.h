@@ -259,6 +259,12 @@ SCOUT_API int scout_sign_chunks_noalloc(uint32_t R, const void *const *replica_p
                                         uint64_t chunk_bytes, scout_sig_t *d_sigs /*device*/,
                                         void *stream);
 
+/* Diagnostic for the fixed array of scout_sign_chunks_noalloc: the array lies between two
+ * 256-byte guard bands that are filled with a pattern when a device is first used; *ok
+ * becomes 1 if both bands still hold it on the current device, 0 if something wrote outside
+ * the array.  Synchronises the device.  Allocates nothing. */
+SCOUT_API int scout_noalloc_guards_ok(int *ok /*host*/);
+
 /* Shape tag for scout_tensor_t.meta_tag: a 64-bit digest of (ndim, dims). */
 SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/);
 
@@ -300,6 +306,11 @@ SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/)
  *                     (asynchronous, so it cannot report) read it here.
  *   set "device_error" 0 clears the flag; a non-zero value sets it from the host
  *                     (a way to exercise the error path without a GPU fault)
+ *   get "debug"       1 if the plan was created with the environment variable SCOUT_DEBUG
+ *                     set to something other than 0: every device buffer the plan owns then
+ *                     lies between two 256-byte guard bands of a fixed pattern
+ *   get "guards_ok"   debug plans only: 1 if no guard band has been written to (synchronises
+ *                     the device); the check that stands in for a memory checker
  *   get "sign_kernels", "certify_kernels"  kernels one scout_sign_chunks / one
  *                     scout_certify call launches for this plan
  *   get "n_tiles", "scratch_bytes", and every settable key

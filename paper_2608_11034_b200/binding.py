@@ -77,6 +77,7 @@ def lib():
             "scout_consensus_vote": (C.c_int, [u32, u64, vp, vp, vp, vp, u64, vp, u64, vp, vp]),
             "scout_consensus_vote_wide": (C.c_int, [u32, u64, vp, u64, u64, vp, vp, vp, u64, vp, u64, vp, vp]),
             "scout_certify": (C.c_int, [vp, vp, vp, vp, u64, vp, u64]),
+            "scout_noalloc_guards_ok": (C.c_int, [vp]),
             "scout_certify_launch": (C.c_int, [vp, vp, u64, u64]),
             "scout_certify_collect": (C.c_int, [vp, vp, vp, u64, vp, u64]),
             "scout_plan_results": (C.c_int, [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)]),
@@ -258,6 +259,13 @@ def scout_sign_chunks_noalloc(R: int, replica_ptrs: Sequence[int], nbytes: int, 
                                            d_sigs, stream), "scout_sign_chunks_noalloc")
 
 
+def scout_noalloc_guards_ok() -> bool:
+    """True if nothing wrote outside the no-allocation entry point's fixed array (synchronises)."""
+    ok = C.c_int(0)
+    _check(lib().scout_noalloc_guards_ok(C.byref(ok)), "scout_noalloc_guards_ok")
+    return bool(ok.value)
+
+
 def scout_consensus_timing(N: int, G: int, d_times: int, kappa: float, d_status: int,
                            d_bitmap: int, d_median: int, d_scale: int, stream: int) -> None:
     _check(lib().scout_consensus_timing(N, G, d_times, kappa, d_status, d_bitmap, d_median,
@@ -386,9 +394,16 @@ def make_tensor_table(specs, tags: Optional[Sequence[int]] = None) -> np.ndarray
 class Plan:
     """Owns a scout plan plus torch-allocated output buffers for sign and vote."""
 
-    def __init__(self, R: int, tensor_table: np.ndarray, chunk_bytes: int):
+    GUARD_BYTES = 256
+    GUARD_PATTERN = 0x5A
+
+    def __init__(self, R: int, tensor_table: np.ndarray, chunk_bytes: int, guards: bool = False):
+        """guards: allocate every output buffer between two 256-byte bands of a fixed pattern;
+        check_guards() then tells whether a kernel wrote outside any of them."""
         import torch
         self._torch = torch
+        self._guards = guards
+        self._outer = []
         self.R, self.T = R, len(tensor_table)
         self.handle = scout_plan_create(R, tensor_table, chunk_bytes)
         self.C = scout_plan_num_chunks(self.handle)
@@ -418,19 +433,39 @@ class Plan:
             out[c] = scout_plan_chunk_info(self.handle, c)
         return out
 
+    def _buffer(self, numel: int, dtype):
+        """A device buffer of `numel` elements; with guards, the middle of a larger one."""
+        torch = self._torch
+        if not self._guards:
+            return torch.empty(numel, dtype=dtype, device="cuda")
+        nbytes = numel * torch.empty(0, dtype=dtype).element_size()
+        g = self.GUARD_BYTES
+        outer = torch.full((nbytes + 2 * g,), self.GUARD_PATTERN, dtype=torch.uint8, device="cuda")
+        self._outer.append((outer, nbytes))
+        return outer[g:g + nbytes].view(dtype)
+
+    def check_guards(self) -> bool:
+        """True if no byte of any guard band has changed (synchronises)."""
+        g = self.GUARD_BYTES
+        self._torch.cuda.synchronize()
+        for outer, nbytes in self._outer:
+            if not bool((outer[:g] == self.GUARD_PATTERN).all()) or \
+                    not bool((outer[g + nbytes:] == self.GUARD_PATTERN).all()):
+                return False
+        return True
+
     def _alloc(self, outlier_cap, undecided_cap):
         torch = self._torch
-        dev = "cuda"
         if self.d_sigs is None:
-            self.d_sigs = torch.empty(self.C * self.R * 32, dtype=torch.uint8, device=dev)
-            self.d_status = torch.empty(max(self.C, 1), dtype=torch.uint8, device=dev)
-            self.d_bitmap = torch.empty(max(self.C, 1), dtype=torch.int64, device=dev)
-            self.d_counts = torch.empty(6, dtype=torch.int64, device=dev)
+            self.d_sigs = self._buffer(self.C * self.R * 32, torch.uint8)
+            self.d_status = self._buffer(max(self.C, 1), torch.uint8)
+            self.d_bitmap = self._buffer(max(self.C, 1), torch.int64)
+            self.d_counts = self._buffer(6, torch.int64)
         if getattr(self, "_ocap", -1) < outlier_cap:
-            self.d_outliers = torch.empty(max(outlier_cap, 1) * 16, dtype=torch.uint8, device=dev)
+            self.d_outliers = self._buffer(max(outlier_cap, 1) * 16, torch.uint8)
             self._ocap = outlier_cap
         if getattr(self, "_ucap", -1) < undecided_cap:
-            self.d_undecided = torch.empty(max(undecided_cap, 1), dtype=torch.int64, device=dev)
+            self.d_undecided = self._buffer(max(undecided_cap, 1), torch.int64)
             self._ucap = undecided_cap
 
     def sign(self, stream: Optional[int] = None) -> None:

@@ -2,6 +2,7 @@
 // validation, launch sequencing, and the certify roll-up.  All arithmetic of the
 // method runs in the kernels of scout_sign.cu and scout_vote.cu.
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -95,6 +96,13 @@ struct scout_plan {
     cudaEvent_t ev_last = nullptr;
     bool launched = false;
 
+    // Debug mode (environment variable SCOUT_DEBUG=1 when the plan is created): every device
+    // buffer the plan owns sits between two guard bands of a fixed byte pattern, and
+    // scout_plan_get(plan, "guards_ok") checks that no kernel wrote into any of them.
+    bool debug = false;
+    struct Guarded { uint8_t *user; size_t bytes; };
+    std::vector<Guarded> guarded;
+
     // optional in-stream timing of the scan kernel (key "timing")
     // a ring of event pairs, one per sign launch, so that a caller can time every launch of a
     // loop and read the durations after it
@@ -104,6 +112,63 @@ struct scout_plan {
 };
 
 namespace {
+
+constexpr size_t GUARD_BYTES = 256;
+constexpr int GUARD_PATTERN = 0xA5;
+
+// Device allocation for a plan.  In debug mode the buffer is preceded and followed by a
+// guard band; the caller gets the address between them (still 256-byte aligned).
+cudaError_t plan_malloc(scout_plan *p, void **ptr, size_t bytes) {
+    if (!p->debug) return cudaMalloc(ptr, bytes);
+    const size_t padded = (bytes + 255) / 256 * 256;   // the rear band starts on a 256-byte boundary
+    uint8_t *base = nullptr;
+    cudaError_t e = cudaMalloc(&base, padded + 2 * GUARD_BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaMemset(base, GUARD_PATTERN, padded + 2 * GUARD_BYTES);
+    if (e != cudaSuccess) {
+        cudaFree(base);
+        return e;
+    }
+    try {
+        p->guarded.push_back({base + GUARD_BYTES, bytes});
+    } catch (const std::bad_alloc &) {
+        cudaFree(base);
+        return cudaErrorMemoryAllocation;
+    }
+    *ptr = base + GUARD_BYTES;
+    return cudaSuccess;
+}
+
+void plan_free(scout_plan *p, void *ptr) {
+    if (!ptr) return;
+    if (p->debug) {
+        for (size_t i = 0; i < p->guarded.size(); ++i)
+            if (p->guarded[i].user == ptr) {
+                p->guarded.erase(p->guarded.begin() + i);
+                cudaFree((uint8_t *)ptr - GUARD_BYTES);
+                return;
+            }
+    }
+    cudaFree(ptr);
+}
+
+// Debug mode: 1 if every guard band of every buffer still holds the pattern.  The bytes
+// between the end of a buffer and the next 256-byte boundary count as guard, too.
+int guards_intact(const scout_plan *p, int64_t *ok) {
+    SCOUT_CUDA(cudaDeviceSynchronize());
+    std::vector<uint8_t> host;
+    *ok = 1;
+    for (const scout_plan::Guarded &g : p->guarded) {
+        const size_t padded = (g.bytes + 255) / 256 * 256;
+        const size_t rear = padded - g.bytes + GUARD_BYTES;
+        host.resize(GUARD_BYTES + rear);
+        SCOUT_CUDA(cudaMemcpy(host.data(), g.user - GUARD_BYTES, GUARD_BYTES, cudaMemcpyDeviceToHost));
+        SCOUT_CUDA(cudaMemcpy(host.data() + GUARD_BYTES, g.user + g.bytes, rear, cudaMemcpyDeviceToHost));
+        for (uint8_t b : host)
+            if (b != (uint8_t)GUARD_PATTERN) *ok = 0;
+    }
+    return SCOUT_OK;
+}
 
 // A plan's tables, scratch and events live on the device that was current when it was
 // created; using it with another device current would launch on the wrong GPU.
@@ -157,13 +222,13 @@ void build_tiles(scout_plan *p) {
 }
 
 int upload_tables(scout_plan *p) {
-    if (p->d_tiles) { cudaFree(p->d_tiles); p->d_tiles = nullptr; }
-    if (p->d_recs) { cudaFree(p->d_recs); p->d_recs = nullptr; }
-    if (p->d_chunks) { cudaFree(p->d_chunks); p->d_chunks = nullptr; }
+    if (p->d_tiles) { plan_free(p, p->d_tiles); p->d_tiles = nullptr; }
+    if (p->d_recs) { plan_free(p, p->d_recs); p->d_recs = nullptr; }
+    if (p->d_chunks) { plan_free(p, p->d_chunks); p->d_chunks = nullptr; }
     const size_t nt = p->tiles.size(), nc = p->chunks.size();
-    SCOUT_CUDA(cudaMalloc(&p->d_tiles, nt * sizeof(TileDesc)));
-    SCOUT_CUDA(cudaMalloc(&p->d_chunks, nc * sizeof(ChunkDesc)));
-    SCOUT_CUDA(cudaMalloc(&p->d_recs, nt * p->R * sizeof(TileRec)));
+    SCOUT_CUDA(plan_malloc(p, (void **)&p->d_tiles, nt * sizeof(TileDesc)));
+    SCOUT_CUDA(plan_malloc(p, (void **)&p->d_chunks, nc * sizeof(ChunkDesc)));
+    SCOUT_CUDA(plan_malloc(p, (void **)&p->d_recs, nt * p->R * sizeof(TileRec)));
     SCOUT_CUDA(cudaMemcpy(p->d_tiles, p->tiles.data(), nt * sizeof(TileDesc), cudaMemcpyHostToDevice));
     SCOUT_CUDA(cudaMemcpy(p->d_chunks, p->chunks.data(), nc * sizeof(ChunkDesc), cudaMemcpyHostToDevice));
     return SCOUT_OK;
@@ -278,26 +343,26 @@ int sign_all(scout_plan *p, cudaStream_t stream, scout_sig_t *d_sigs, CertifyOut
 int ensure_certify_buffers(scout_plan *p, uint64_t outlier_cap, uint64_t undecided_cap) {
     const uint64_t C = p->chunks.size();
     if (!p->d_sigs) {
-        SCOUT_CUDA(cudaMalloc(&p->d_sigs, C * p->R * sizeof(scout_sig_t)));
-        SCOUT_CUDA(cudaMalloc(&p->d_status, C));
-        SCOUT_CUDA(cudaMalloc(&p->d_bitmap, C * sizeof(uint64_t)));
-        SCOUT_CUDA(cudaMalloc(&p->d_majority, C * sizeof(uint64_t)));
-        SCOUT_CUDA(cudaMalloc(&p->d_out, sizeof(CertifyOut)));
+        SCOUT_CUDA(plan_malloc(p, (void **)&p->d_sigs, C * p->R * sizeof(scout_sig_t)));
+        SCOUT_CUDA(plan_malloc(p, (void **)&p->d_status, C));
+        SCOUT_CUDA(plan_malloc(p, (void **)&p->d_bitmap, C * sizeof(uint64_t)));
+        SCOUT_CUDA(plan_malloc(p, (void **)&p->d_majority, C * sizeof(uint64_t)));
+        SCOUT_CUDA(plan_malloc(p, (void **)&p->d_out, sizeof(CertifyOut)));
         SCOUT_CUDA(cudaMemset(p->d_out, 0, sizeof(CertifyOut)));
         SCOUT_CUDA(cudaHostAlloc(&p->h_out, sizeof(CertifyHost), cudaHostAllocMapped));
         SCOUT_CUDA(cudaHostGetDevicePointer((void **)&p->h_out_dev, p->h_out, 0));
     }
     if (!p->d_outliers || outlier_cap > p->outlier_cap) {
-        if (p->d_outliers) cudaFree(p->d_outliers);
+        if (p->d_outliers) plan_free(p, p->d_outliers);
         p->d_outliers = nullptr;
         p->outlier_cap = std::max<uint64_t>(outlier_cap, 1);
-        SCOUT_CUDA(cudaMalloc(&p->d_outliers, p->outlier_cap * sizeof(scout_outlier_t)));
+        SCOUT_CUDA(plan_malloc(p, (void **)&p->d_outliers, p->outlier_cap * sizeof(scout_outlier_t)));
     }
     if (!p->d_undecided || undecided_cap > p->undecided_cap) {
-        if (p->d_undecided) cudaFree(p->d_undecided);
+        if (p->d_undecided) plan_free(p, p->d_undecided);
         p->d_undecided = nullptr;
         p->undecided_cap = std::max<uint64_t>(undecided_cap, 1);
-        SCOUT_CUDA(cudaMalloc(&p->d_undecided, p->undecided_cap * sizeof(uint64_t)));
+        SCOUT_CUDA(plan_malloc(p, (void **)&p->d_undecided, p->undecided_cap * sizeof(uint64_t)));
     }
     return SCOUT_OK;
 }
@@ -423,6 +488,8 @@ int scout_plan_create(uint32_t R, uint64_t T, const scout_tensor_t *tensors, uin
     p->R = R;
     p->T = T;
     p->chunk_bytes = chunk_bytes;
+    const char *dbg = std::getenv("SCOUT_DEBUG");
+    p->debug = dbg && dbg[0] && dbg[0] != '0';
     uint64_t total = 0, poff = 0;
     try {
         p->tensors.assign(tensors, tensors + T);
@@ -473,19 +540,19 @@ int scout_plan_create(uint32_t R, uint64_t T, const scout_tensor_t *tensors, uin
         if (cudaGetDevice(&p->device) != cudaSuccess) { rc = SCOUT_ERR_CUDA; break; }
         if ((rc = sign_grid_size(p->variant, p->uniform_dtype, p->device, &p->grid))) break;
         if ((rc = upload_tables(p))) break;
-        if (cudaMalloc(&p->d_tensor_chunk0, (T + 1) * sizeof(uint64_t)) != cudaSuccess ||
-            cudaMalloc(&p->d_ptrs, (size_t)R * T * sizeof(void *)) != cudaSuccess ||
-            cudaMalloc(&p->d_error, sizeof(uint32_t)) != cudaSuccess) {
+        if (plan_malloc(p, (void **)&p->d_tensor_chunk0, (T + 1) * sizeof(uint64_t)) != cudaSuccess ||
+            plan_malloc(p, (void **)&p->d_ptrs, (size_t)R * T * sizeof(void *)) != cudaSuccess ||
+            plan_malloc(p, (void **)&p->d_error, sizeof(uint32_t)) != cudaSuccess) {
             rc = SCOUT_ERR_NOMEM;
             break;
         }
         const size_t nc = p->chunks.size();
         const size_t n_tickets = nc * R + nc;  // one per (chunk, replica), then one per chunk
-        if (cudaMalloc(&p->d_tickets, n_tickets * sizeof(uint32_t)) != cudaSuccess ||
-            cudaMalloc(&p->d_done, nc * sizeof(uint32_t)) != cudaSuccess ||
-            cudaMalloc(&p->d_chain, sizeof(ChainState)) != cudaSuccess ||
-            cudaMalloc(&p->d_work, 2 * sizeof(unsigned long long)) != cudaSuccess ||
-            cudaMalloc(&p->d_work2, 2 * sizeof(unsigned long long)) != cudaSuccess) {
+        if (plan_malloc(p, (void **)&p->d_tickets, n_tickets * sizeof(uint32_t)) != cudaSuccess ||
+            plan_malloc(p, (void **)&p->d_done, nc * sizeof(uint32_t)) != cudaSuccess ||
+            plan_malloc(p, (void **)&p->d_chain, sizeof(ChainState)) != cudaSuccess ||
+            plan_malloc(p, (void **)&p->d_work, 2 * sizeof(unsigned long long)) != cudaSuccess ||
+            plan_malloc(p, (void **)&p->d_work2, 2 * sizeof(unsigned long long)) != cudaSuccess) {
             rc = SCOUT_ERR_NOMEM;
             break;
         }
@@ -552,27 +619,27 @@ int scout_plan_chunk_info(const scout_plan_t *p, uint64_t c, uint64_t *tensor, u
 
 int scout_plan_destroy(scout_plan_t *p) {
     if (!p) return SCOUT_OK;
-    cudaFree(p->d_tiles);
-    cudaFree(p->d_chunks);
-    cudaFree(p->d_tensor_chunk0);
-    cudaFree((void *)p->d_ptrs);
-    cudaFree(p->d_recs);
-    cudaFree(p->d_error);
-    cudaFree(p->d_tickets);
-    cudaFree(p->d_done);
-    cudaFree(p->d_chain);
-    cudaFree(p->d_work);
-    cudaFree(p->d_work2);
-    cudaFree(p->d_sigs);
-    cudaFree(p->d_status);
-    cudaFree(p->d_bitmap);
-    cudaFree(p->d_majority);
-    cudaFree(p->d_undecided);
-    cudaFree(p->d_outliers);
-    cudaFree(p->d_out);
+    plan_free(p, p->d_tiles);
+    plan_free(p, p->d_chunks);
+    plan_free(p, p->d_tensor_chunk0);
+    plan_free(p, (void *)p->d_ptrs);
+    plan_free(p, p->d_recs);
+    plan_free(p, p->d_error);
+    plan_free(p, p->d_tickets);
+    plan_free(p, p->d_done);
+    plan_free(p, p->d_chain);
+    plan_free(p, p->d_work);
+    plan_free(p, p->d_work2);
+    plan_free(p, p->d_sigs);
+    plan_free(p, p->d_status);
+    plan_free(p, p->d_bitmap);
+    plan_free(p, p->d_majority);
+    plan_free(p, p->d_undecided);
+    plan_free(p, p->d_outliers);
+    plan_free(p, p->d_out);
     if (p->h_out) cudaFreeHost(p->h_out);
     for (int i = 0; i < 2; ++i) {
-        cudaFree(p->d_stage[i]);
+        plan_free(p, p->d_stage[i]);
         if (p->ev_copied[i]) cudaEventDestroy(p->ev_copied[i]);
         if (p->ev_done[i]) cudaEventDestroy(p->ev_done[i]);
     }
@@ -673,7 +740,7 @@ int scout_certify_host(scout_plan_t *p, const void *const *h_ptrs, scout_report_
         }
         p->stage_bytes = std::min<uint64_t>(packed, 256ull << 20);
         p->stage_bytes = std::max<uint64_t>(p->stage_bytes, (uint64_t)p->tile_bytes + 256);
-        for (int i = 0; i < 2; ++i) SCOUT_CUDA(cudaMalloc(&p->d_stage[i], p->stage_bytes));
+        for (int i = 0; i < 2; ++i) SCOUT_CUDA(plan_malloc(p, (void **)&p->d_stage[i], p->stage_bytes));
     }
     const uint64_t NT = p->tiles.size();
     uint64_t slice = 0;
@@ -798,7 +865,7 @@ int scout_plan_set(scout_plan_t *p, const char *key, int64_t value) {
             return SCOUT_ERR_NOMEM;
         }
         if (p->d_stage[0]) {  // staging was sized for the old tiles
-            for (int i = 0; i < 2; ++i) { cudaFree(p->d_stage[i]); p->d_stage[i] = nullptr; }
+            for (int i = 0; i < 2; ++i) { plan_free(p, p->d_stage[i]); p->d_stage[i] = nullptr; }
             cudaStreamDestroy(p->s_copy);
             cudaStreamDestroy(p->s_comp);
             p->s_copy = p->s_comp = nullptr;
@@ -856,6 +923,12 @@ int scout_plan_get(const scout_plan_t *p, const char *key, int64_t *value) {
     else if (!std::strcmp(key, "variant")) *value = p->variant;
     else if (!std::strcmp(key, "grid")) *value = p->grid;
     else if (!std::strcmp(key, "n_tiles")) *value = (int64_t)p->tiles.size();
+    else if (!std::strcmp(key, "debug")) *value = p->debug;
+    else if (!std::strcmp(key, "guards_ok")) {
+        if (!p->debug) return SCOUT_ERR_INVALID;  // there are no guard bands to look at
+        if (int rc = check_device(p)) return rc;
+        return guards_intact(p, value);
+    }
     else if (!std::strcmp(key, "fused")) *value = p->fused;
     else if (!std::strcmp(key, "dynamic")) *value = p->dynamic;
     else if (!std::strcmp(key, "sign_kernels")) *value = use_fused(p, false) ? 1 : 2;    // scan, finalise

@@ -1565,7 +1565,12 @@ constexpr uint32_t NOALLOC_MAX_DEVICES = 64;
 // The scratch itself.  In host code this name is only a stand-in for the
 // symbol, not an address a kernel can use; the host obtains the device address
 // with cudaGetSymbolAddress (below) and passes that to the kernels.
-static __device__ __align__(256) TileRec g_noalloc_scratch[NOALLOC_MAX_RECORDS];
+// Eight records (256 bytes) of guard band on either side: they are filled with a pattern at
+// set-up and scout_noalloc_guards_ok() checks that no kernel has written to them.
+constexpr uint32_t NOALLOC_GUARD_RECORDS = 8;
+constexpr int NOALLOC_GUARD_PATTERN = 0xC3;
+static __device__ __align__(256) TileRec g_noalloc_scratch[NOALLOC_GUARD_RECORDS + NOALLOC_MAX_RECORDS +
+                                                           NOALLOC_GUARD_RECORDS];
 
 struct NoallocArgs {
     const uint8_t *replica[64];
@@ -1642,7 +1647,11 @@ int noalloc_setup(int device, NoallocDevice *out) {
         SCOUT_CUDA(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
         int sms = 0;
         SCOUT_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
-        d.scratch = static_cast<TileRec *>(ptr);
+        TileRec *base = static_cast<TileRec *>(ptr);
+        SCOUT_CUDA(cudaMemset(base, NOALLOC_GUARD_PATTERN, NOALLOC_GUARD_RECORDS * sizeof(TileRec)));
+        SCOUT_CUDA(cudaMemset(base + NOALLOC_GUARD_RECORDS + NOALLOC_MAX_RECORDS, NOALLOC_GUARD_PATTERN,
+                              NOALLOC_GUARD_RECORDS * sizeof(TileRec)));
+        d.scratch = base + NOALLOC_GUARD_RECORDS;
         d.sms = sms;
         d.ready = true;
     }
@@ -1652,6 +1661,25 @@ int noalloc_setup(int device, NoallocDevice *out) {
 
 }  // namespace
 }  // namespace scout
+
+extern "C" int scout_noalloc_guards_ok(int *ok) {
+    using namespace scout;
+    if (!ok) return SCOUT_ERR_INVALID;
+    int device = 0;
+    SCOUT_CUDA(cudaGetDevice(&device));
+    NoallocDevice dev;
+    int rc = noalloc_setup(device, &dev);
+    if (rc) return rc;
+    SCOUT_CUDA(cudaDeviceSynchronize());
+    uint8_t host[2 * NOALLOC_GUARD_RECORDS * sizeof(TileRec)];
+    const size_t band = NOALLOC_GUARD_RECORDS * sizeof(TileRec);
+    SCOUT_CUDA(cudaMemcpy(host, dev.scratch - NOALLOC_GUARD_RECORDS, band, cudaMemcpyDeviceToHost));
+    SCOUT_CUDA(cudaMemcpy(host + band, dev.scratch + NOALLOC_MAX_RECORDS, band, cudaMemcpyDeviceToHost));
+    *ok = 1;
+    for (uint8_t b : host)
+        if (b != (uint8_t)NOALLOC_GUARD_PATTERN) *ok = 0;
+    return SCOUT_OK;
+}
 
 extern "C" int scout_sign_chunks_noalloc(uint32_t R, const void *const *replica_ptrs, uint64_t nbytes,
                                          uint32_t dtype, uint64_t meta_tag, uint64_t chunk_bytes,

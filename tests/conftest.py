@@ -9,6 +9,12 @@ for p in (ROOT, os.path.join(ROOT, "tests")):
         sys.path.insert(0, p)
 
 
+# Plans created by the tests run in the library's debug mode: every device buffer a plan owns
+# is allocated between guard bands, which the helpers check after each run (the stand-in for
+# a memory checker on machines where none may be run).
+os.environ.setdefault("SCOUT_DEBUG", "1")
+
+
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (runs on the B200 box only)")
 

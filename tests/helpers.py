@@ -64,8 +64,9 @@ def expected_from_patches(w, chunks):
 def gpu_plan(w, chunk_bytes=None, tags=None, tile_bytes=None, variant=None):
     from paper_2608_11034_b200 import binding
     tags = shape_tags(w) if tags is None else tags
+    # every output buffer of the tests sits between guard bands (see gpu_sign_vote)
     plan = binding.Plan(w.R, binding.make_tensor_table(w.specs, tags),
-                        w.chunk_bytes if chunk_bytes is None else chunk_bytes)
+                        w.chunk_bytes if chunk_bytes is None else chunk_bytes, guards=True)
     if tile_bytes is not None:
         binding.scout_plan_set(plan.handle, "tile_bytes", tile_bytes)
     if variant == "unfused":      # the default scan, one kernel per stage
@@ -86,8 +87,21 @@ def gpu_sign_vote(w, views, chunk_bytes=None, tags=None, tile_bytes=None, caps=(
     plan.sign_and_vote(*caps)
     out = plan.fetch()
     assert binding.scout_plan_get(plan.handle, "device_error") == 0
+    # nothing was written outside the caller's output buffers, nor (debug mode, which the GPU
+    # tests switch on through SCOUT_DEBUG=1) outside any buffer the plan owns
+    assert plan.check_guards()
+    if binding.scout_plan_get(plan.handle, "debug"):
+        assert binding.scout_plan_get(plan.handle, "guards_ok") == 1
     plan.close()
     return out
+
+
+def assert_guards(plan):
+    """No kernel wrote outside the caller's output buffers nor outside the plan's own."""
+    from paper_2608_11034_b200 import binding
+    assert plan.check_guards()
+    if binding.scout_plan_get(plan.handle, "debug"):
+        assert binding.scout_plan_get(plan.handle, "guards_ok") == 1
 
 
 def chunk_abs_sums(w, views, chunks):

@@ -43,6 +43,7 @@ def test_plan_knobs():
     assert B.scout_plan_get(h, "last_sign_ns") > 0 and B.scout_plan_get(h, "device_error") == 0
     ref = helpers.gpu_sign_vote(w, views)
     assert (got["sigs"]["hash"] == ref["sigs"]["hash"]).all() and got["outliers"] == ref["outliers"]
+    helpers.assert_guards(plan)
     plan.close()
 
 
@@ -67,6 +68,7 @@ def test_rebinding_and_user_streams():
     assert (results[0]["sigs"]["hash"] != results[1]["sigs"]["hash"]).all()
     rep = plan.certify(stream=side.cuda_stream)
     assert rep["outliers"] == results[0]["outliers"]
+    helpers.assert_guards(plan)
     plan.close()
 
 
@@ -99,6 +101,7 @@ def test_certify_host_with_pageable_and_scattered_tensors():
     plan.bind(dviews)
     got3 = plan.certify()
     assert got3["report"] == want["report"]
+    helpers.assert_guards(plan)
     plan.close()
 
 
@@ -146,6 +149,7 @@ def test_device_error_flag_is_reported_once_and_cleared():
     assert B.scout_plan_get(plan.handle, "device_error") == 1
     B.scout_plan_set(plan.handle, "device_error", 0)
     assert B.scout_plan_get(plan.handle, "device_error") == 0
+    helpers.assert_guards(plan)
     plan.close()
 
 
@@ -171,6 +175,7 @@ def test_rebinding_waits_for_a_scan_in_flight_on_a_non_blocking_stream():
     side.synchronize()
     got_a = d_a.cpu().numpy().view(B.SIG_DTYPE).reshape(plan.C, wa.R)
     got_b = d_b.cpu().numpy().view(B.SIG_DTYPE).reshape(plan.C, wa.R)
+    helpers.assert_guards(plan)
     plan.close()
     ref_a = helpers.gpu_sign_vote(wa, va)["sigs"]
     ref_b = helpers.gpu_sign_vote(wb, vb)["sigs"]
@@ -188,6 +193,7 @@ def test_a_plan_used_with_another_device_current_is_rejected():
     plan = helpers.gpu_plan(w)
     plan.bind(views)
     if torch.cuda.device_count() < 2:
+        helpers.assert_guards(plan)
         plan.close()
         pytest.skip("needs two GPUs")
     d_sigs = torch.zeros(plan.C * w.R * 32, dtype=torch.uint8, device="cuda:0")
@@ -200,4 +206,28 @@ def test_a_plan_used_with_another_device_current_is_rejected():
             B.scout_plan_bind(plan.handle, [v.data_ptr() for rep in views for v in rep])
     finally:
         torch.cuda.set_device(0)
+    helpers.assert_guards(plan)
+    plan.close()
+
+
+def test_guard_bands_notice_a_stray_write():
+    """The tests' stand-in for a memory checker: output buffers between guard bands.  A byte
+    written just outside a buffer (here by hand) is reported; untouched bands are not."""
+    from paper_2608_11034_b200 import binding as B
+    w = inputs.workload(1, "default", 1 / 16)
+    _, views = inputs.generate(w, "cuda")
+    plan = helpers.gpu_plan(w)
+    assert B.scout_plan_get(plan.handle, "debug") == 1      # conftest switches the debug mode on
+    plan.bind(views)
+    plan.sign_and_vote()
+    plan.certify()
+    helpers.assert_guards(plan)
+    outer, nbytes = plan._outer[0]
+    outer[B.Plan.GUARD_BYTES + nbytes] = 0                   # first byte after the record table
+    assert not plan.check_guards()
+    outer[B.Plan.GUARD_BYTES + nbytes] = B.Plan.GUARD_PATTERN
+    outer[B.Plan.GUARD_BYTES - 1] = 1                        # last byte before it
+    assert not plan.check_guards()
+    outer[B.Plan.GUARD_BYTES - 1] = B.Plan.GUARD_PATTERN
+    assert plan.check_guards()
     plan.close()

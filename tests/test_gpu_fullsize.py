@@ -176,6 +176,7 @@ def test_config_4_certify_full_size():
     maj = [int(sigs["hash"][c, (bad + 1) % w.R]) for c in range(plan.C)]
     import defn
     assert r["certificate"] == defn.certificate(maj)
+    helpers.assert_guards(plan)
     plan.close()
     del views
     _free()
@@ -201,6 +202,7 @@ def test_config_5_full_size():
     assert (sigs["hash"][clean] == sigs["hash"][clean][:, :1]).all()
     _check_sampled(w, views, sigs, chunks, _sample_pairs(w, chunks, want_out, 40, 5))
     _check_whole_replica(w, views, sigs, chunks, want_out[0][1])
+    helpers.assert_guards(plan)
     plan.close()
     del views
     _free()
@@ -232,6 +234,7 @@ def test_config_3_full_size():
     assert (sigs["hash"][clean] == sigs["hash"][clean][:, :1]).all()
     _check_sampled(w, views, sigs, chunks, _sample_pairs(w, chunks, want_out, 8, 3))
     _check_whole_replica(w, views, sigs, chunks, 5)
+    helpers.assert_guards(plan)
     plan.close()
     del views
     _free()
@@ -259,6 +262,7 @@ def test_largest_chunk_size_one_gib():
     assert got["outliers"] == [] and got["undecided"] == [0, 3]
     assert list(got["status"]) == [binding.INCONCLUSIVE, binding.AGREE, binding.AGREE, binding.INCONCLUSIVE]
     _check_sampled(w, views, got["sigs"], chunks, [(0, 1), (1, 0), (2, 0), (3, 0), (3, 1)])
+    helpers.assert_guards(plan)
     plan.close()
     del views
     _free()

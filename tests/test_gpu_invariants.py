@@ -28,6 +28,7 @@ def test_thirty_clean_runs_stay_clean_and_identical():
         blob = got["sigs"].tobytes()
         first = first or blob
         assert blob == first
+    helpers.assert_guards(plan)
     plan.close()
 
 
@@ -94,4 +95,5 @@ def test_every_bit_of_an_element_is_seen(dtype):
     assert len(seen) == 8 * es
     plan.sign_and_vote()
     assert plan.fetch()["outliers"] == []
+    helpers.assert_guards(plan)
     plan.close()

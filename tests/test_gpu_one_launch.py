@@ -63,6 +63,7 @@ def test_certify_in_one_launch_equals_the_oracle_and_the_staged_form(cfg, case, 
     B.scout_plan_set(plan.handle, "fused", 1)
     again = plan.certify()
     assert again["report"] == want["report"] and again["outliers"] == want["outliers"]
+    helpers.assert_guards(plan)
     plan.close()
 
 
@@ -89,6 +90,7 @@ def test_lists_longer_than_the_report_head_and_truncation():
     assert len(cut["undecided"]) == 3 and set(cut["undecided"]) <= set(want["undecided"])
     full = plan.certify()
     assert full["outliers"] == want["outliers"] and full["undecided"] == want["undecided"]
+    helpers.assert_guards(plan)
     plan.close()
 
 
@@ -113,6 +115,7 @@ def test_launch_and_collect():
         assert got["report"] == want["report"] and got["outliers"] == want["outliers"]
         with pytest.raises(B.ScoutError):                  # already collected
             plan.certify_collect()
+    helpers.assert_guards(plan)
     plan.close()
 
 
@@ -140,4 +143,5 @@ def test_sign_in_one_launch_with_one_replica_and_with_sixty_four():
             want = orc.certify(osigs)
             assert got["report"] == want["report"] and got["outliers"] == want["outliers"]
             assert got["report"]["replica_union_bitmap"] == (1 << 63) | (1 << 31) | (1 << 32)
+        helpers.assert_guards(plan)
         plan.close()

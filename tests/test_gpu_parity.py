@@ -248,6 +248,7 @@ def test_certify_and_rollups():
         sel = np.nonzero(chunks["tensor"] == t)[0]
         for r in range(w.R):
             assert int(roll[t, r]) == orc.rollup(osigs["hash"][sel, r])
+    helpers.assert_guards(plan)
     plan.close()
 
     # clean and undecided verdicts
@@ -263,6 +264,7 @@ def test_certify_and_rollups():
     rep = plan.certify()
     assert rep["report"]["verdict"] == b.UNDECIDED and rep["report"]["certificate"] == 0
     assert len(rep["undecided"]) == 1 and rep["outliers"] == []
+    helpers.assert_guards(plan)
     plan.close()
 
 
@@ -278,6 +280,7 @@ def test_certify_host_streams_pinned_replicas():
     got = b.scout_certify_host(plan.handle, [v.data_ptr() for rep in pviews for v in rep])
     assert got["report"] == want["report"] and got["outliers"] == want["outliers"]
     d_sigs, _, _ = b.scout_plan_results(plan.handle)
+    helpers.assert_guards(plan)
     plan.close()
 
 
@@ -293,6 +296,7 @@ def test_bind_rejects_misaligned_and_null_pointers():
         assert e.value.code == code
     with pytest.raises(b.ScoutError):           # signing before a successful bind
         plan.sign()
+    helpers.assert_guards(plan)
     plan.close()
 
 
@@ -311,4 +315,5 @@ def test_three_step_protocol_clean_fault_clean():
     inputs.revert_patches(views, w.specs, w.patches, old)
     plan.sign_and_vote()
     assert plan.fetch()["outliers"] == []
+    helpers.assert_guards(plan)
     plan.close()

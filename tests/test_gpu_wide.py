@@ -117,4 +117,5 @@ def test_signing_more_than_64_replicas():
     with pytest.raises(B.ScoutError) as e:
         plan.certify()
     assert e.value.code == B.ERR_UNSUPPORTED
+    helpers.assert_guards(plan)
     plan.close()

@@ -57,6 +57,7 @@ def _noalloc(w, views):
     torch.cuda.synchronize()
     host = d_sigs.cpu().numpy()
     assert (host[C * w.R * 32:] == 0xAB).all(), "write past the end of the record table"
+    assert binding.scout_noalloc_guards_ok(), "write outside the fixed scratch array"
     return host[:C * w.R * 32].view(binding.SIG_DTYPE).reshape(C, w.R)
 
 
