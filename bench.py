@@ -37,11 +37,32 @@ NOMINAL_HBM_GBS = 8000.0
 BENCH_CASE = {2: "mantissa"}   # config 2 is timed on its one-flip case, so every config carries a fault
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) per algorithmic byte of the scan kernel, from the ncu
-# captures summarised under profiles/: 1.8007 GB read + 0.026 GB written for
-# 1.8000 GB scanned (fp32), 1.1407 + 0.016 for 1.1401 GB (bf16).  Traffic grows
-# in proportion to the bytes scanned, so a full-size launch is scaled by this.
-SCAN_TRAFFIC_RATIO = 1.0148
-SCAN_TRAFFIC_SOURCE = "ncu capture of the scan kernel on 1.8 GB, scaled to the launch (profiles/)"
+# captures summarised under profiles/: 1.8006 GB read + 0.0264 GB written for
+# 1.8000 GB scanned (fp32), 4.5996 + 0.020 for 4.5993 GB (bf16, ratio 1.0045).  Traffic
+# grows in proportion to the bytes scanned, so a full-size launch is scaled by this.
+# To be measured again whenever the scan kernel changes.
+SCAN_TRAFFIC_RATIO = 1.0150
+SCAN_TRAFFIC_SOURCE = ("ncu capture of the scan kernel on 1.8 GB at commit 1975673, scaled to the launch "
+                       "(profiles/sign_tiles_direct_fp32_and_bf16.md section 2)")
+
+
+# SM cycles per 512-byte row and scheduler of the scan's row routine with its data already on the
+# SM (profiles/row_routine_issue_bound.md, `python -m paper_2608_11034_b200.microbench`): the
+# compute bound of a uniform-dtype workload at SM clock f is 512 B * 4 * SMs * f / cycles.
+ROW_COST_CYCLES = {"bf16": 81.4, "f16": 81.3, "f32": 51.4, "i64": 41.3, "u8": 26.9}
+N_SMS = 148
+
+
+def compute_bound(w, clocks, value):
+    """The scan rate the row routine allows at the SM clock sampled during the timed region."""
+    dtypes = {s.dtype for s in w.specs}
+    if len(dtypes) != 1 or next(iter(dtypes)) not in ROW_COST_CYCLES or not clocks or not clocks.get("sm_mhz"):
+        return None
+    cyc = ROW_COST_CYCLES[next(iter(dtypes))]
+    bound = 512 * 4 * N_SMS * clocks["sm_mhz"] * 1e6 / cyc / 1e9
+    return {"bound": "alu", "cycles_per_row_per_scheduler": cyc, "sm_mhz_sampled": clocks["sm_mhz"],
+            "bound_gbs": bound, "frac": value / bound,
+            "source": "row_cost microbenchmark (profiles/row_routine_issue_bound.md)"}
 
 
 def measured_peak():
@@ -413,7 +434,7 @@ def run_config(cfg, args, rank, world, local, headline):
         "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
         "frac_of_measured_copy": value / world / peak,
         "verified": True, "verdict": verdict, "clocks": clocks, "roofline": roofline, "l2_warm": warm,
-        "one_launch": one_launch,
+        "one_launch": one_launch, "compute_bound": compute_bound(w, clocks, value) if world == 1 else None,
     }
 
     # ---- end to end: replicas in pinned host memory, copies inside the timed region
@@ -551,7 +572,7 @@ def main():
         "verified": head["verified"], "verdict": head["verdict"],
         "gpu_launches": head["launch"]["kernels_per_step"] * args.steps,
         "clocks": head["clocks"], "roofline": head["roofline"], "l2_warm": head["l2_warm"],
-        "one_launch": head["one_launch"],
+        "one_launch": head["one_launch"], "compute_bound": head["compute_bound"],
         "e2e": head["e2e"], "cpu_baseline": head["cpu_baseline"],
     }
 
@@ -573,6 +594,7 @@ def main():
                                                           "scan_share_of_step_time", "read_probe_gbs",
                                                           "frac_of_read_probe")},
                 "clocks": r["clocks"], "verified": r["verified"], "regime": r["launch"]["regime"],
+                "tile_bytes": r["launch"]["tile_bytes"], "compute_bound": r["compute_bound"],
                 "parity_spot_check": (r["cpu_baseline"] or {}).get("parity_spot_check"),
                 "cpu_oracle_gbs": (r["cpu_baseline"] or {}).get("value"),
             }
