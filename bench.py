@@ -326,7 +326,7 @@ def run_config(cfg, args, rank, world, local, headline):
     dist_util.barrier()
     clocks = sampler.stop() if sampler else None
     step_ms = [a.elapsed_time(b) for a, b in ev]
-    ms = dist_util.max_over_ranks(sum(step_ms), "cuda")
+    ms = dist_util.max_over_ranks(sum(step_ms), dist_util.reduce_device())
     n_scan = binding.scout_plan_get(plan.handle, "timed_sign_launches")
     scan_ns = binding.scout_plan_get(plan.handle, "timed_sign_ns")
     # the ring holds the last 256 launches: with more steps than that, compare like with like
@@ -528,7 +528,7 @@ def run_distributed(args, rank, world, local):
         a.record(); c3.step(); b.record()
     torch.cuda.synchronize()
     dist_util.barrier()
-    ms = dist_util.max_over_ranks(sum(a.elapsed_time(b) for a, b in ev), "cuda")
+    ms = dist_util.max_over_ranks(sum(a.elapsed_time(b) for a, b in ev), dist_util.reduce_device())
     got = c3.fetch()
     # chunks that hold a patch must be the ones named (attributed with R >= 3; with R = 2 a
     # difference cannot be attributed and the chunk is listed as undecided)
@@ -537,10 +537,12 @@ def run_distributed(args, rank, world, local):
     named = sorted({c for c, _ in got["outliers"]} | set(got["undecided"]))
     if named != want:
         raise SystemExit(f"distributed C3: chunks named {named}, expected {want}")
+    n_chunks, on_device = c3.C, c3.device_transport
     c3.close()
     return {"value": world * w.bytes_per_replica * args.steps / (ms * 1e-3) / 1e9, "unit": UNIT,
             "ms_per_step": ms / args.steps, "R": world, "bytes_per_rank_per_step": w.bytes_per_replica,
-            "gathered_bytes_per_rank": c3.C * 32, "transport": "nccl all_gather_into_tensor",
+            "gathered_bytes_per_rank": n_chunks * 32,
+            "transport": "nccl all_gather_into_tensor" if on_device else "host all_gather (gloo)",
             "chunks_named": named, "form": "one replica per GPU: sign, all-gather records, vote on every rank"}
 
 
@@ -556,9 +558,14 @@ def main():
     rank, world, local = dist_util.rank_info()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (the product path has no CPU fallback)")
+    # Test hook for boxes with one GPU: every rank uses cuda:0 and the ranks talk over gloo, so the
+    # N > 1 code path (barrier, max over ranks, distributed C3) can run; its numbers mean nothing.
+    one_gpu = os.environ.get("SCOUT_BENCH_ALL_RANKS_ON_GPU0") == "1"
+    if one_gpu:
+        local = 0
     torch.cuda.set_device(local)
     if world > 1:
-        dist_util.init("nccl", torch.device("cuda", local))
+        dist_util.init("gloo" if one_gpu else "nccl", torch.device("cuda", local))
 
     head = run_config(args.config, args, rank, world, local, headline=True)
     line = {

@@ -34,6 +34,13 @@ def barrier() -> None:
         dist.barrier()
 
 
+def reduce_device() -> str:
+    """Where the tensors of the small cross-rank reductions live: the GPU under NCCL."""
+    if dist.is_available() and dist.is_initialized() and dist.get_backend() == "nccl":
+        return "cuda"
+    return "cpu"
+
+
 def max_over_ranks(value: float, device="cpu") -> float:
     if not (dist.is_available() and dist.is_initialized()):
         return float(value)

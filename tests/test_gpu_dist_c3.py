@@ -86,3 +86,25 @@ def test_three_ranks_agree_with_the_fused_path_and_the_oracle(world):
     want = orc.vote(osigs)
     assert outliers == want["outliers"] == helpers.expected_from_patches(w, chunks)[0] and len(outliers) == 2
     assert undecided == want["undecided"] == []
+
+
+def test_bench_multi_rank_path_runs_on_one_gpu():
+    """`bench.py --gpus 2` through the launcher, with both ranks on cuda:0 and gloo between them
+    (a test hook of bench.py): the barrier, the max over ranks and the distributed-C3 leg run and
+    rank 0 prints one JSON line.  The numbers mean nothing; the code path is what is checked."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, SCOUT_BENCH_ALL_RANKS_ON_GPU0="1")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
+           "--master-addr", "127.0.0.1", "--master-port", str(_free_port()), os.path.join(root, "bench.py"),
+           "--gpus", "2", "--steps", "2", "--warmup", "1", "--scale", "0.002", "--no-e2e", "--no-cpu-baseline"]
+    out = subprocess.run(cmd, capture_output=True, text=True, timeout=600, env=env, cwd=root)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["verified"] and line["scaling"] == "weak"
+    d = line["distributed_c3"]
+    assert d["R"] == 2 and d["value"] > 0 and len(d["chunks_named"]) >= 1
