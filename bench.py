@@ -43,11 +43,11 @@ FALLBACK_HBM_GBS = 6650.0
 # To be measured again whenever the scan kernel changes.
 SCAN_TRAFFIC_RATIO = 1.0150
 SCAN_TRAFFIC_SOURCE = ("ncu capture of the scan kernel on 1.8 GB at commit 1975673, scaled to the launch "
-                       "(profiles/sign_tiles_direct_fp32_and_bf16.md section 2)")
+                       "(summary under profiles/)")
 
 
 # SM cycles per 512-byte row and scheduler of the scan's row routine with its data already on the
-# SM (profiles/row_routine_issue_bound.md, `python -m paper_2608_11034_b200.microbench`): the
+# SM (`python -m paper_2608_11034_b200.microbench`, its output is summarised under profiles/): the
 # compute bound of a uniform-dtype workload at SM clock f is 512 B * 4 * SMs * f / cycles.
 ROW_COST_CYCLES = {"bf16": 81.4, "f16": 81.3, "f32": 51.4, "i64": 41.3, "u8": 26.9}
 N_SMS = 148
@@ -62,7 +62,7 @@ def compute_bound(w, clocks, value):
     bound = 512 * 4 * N_SMS * clocks["sm_mhz"] * 1e6 / cyc / 1e9
     return {"bound": "alu", "cycles_per_row_per_scheduler": cyc, "sm_mhz_sampled": clocks["sm_mhz"],
             "bound_gbs": bound, "frac": value / bound,
-            "source": "row_cost microbenchmark (profiles/row_routine_issue_bound.md)"}
+            "source": "row_cost microbenchmark (python -m paper_2608_11034_b200.microbench)"}
 
 
 def measured_peak():
