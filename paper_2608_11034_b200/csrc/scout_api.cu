@@ -242,8 +242,8 @@ int upload_tables(scout_plan *p) {
 //     7.2 TB/s on 36 GB of fp32 and 6.25 TB/s on 125 GB of bf16; the one-launch kernel, whose
 //     loop also carries the ticket state (it spills) and takes tiles replica-interleaved, stays
 //     3 to 7 % below that, more than the three small launches it saves.  What the one-launch
-//     form alone offers at large sizes is the certificate chain folded behind the scan (39 ns
-//     per chunk otherwise: 28 us at 717 chunks, 0.9 ms at 24,000).
+//     form alone offers at large sizes is the certificate chain folded behind the scan (32 ns
+//     per chunk otherwise: 23 us at 717 chunks, 0.8 ms at 24,000).
 bool use_fused(const scout_plan *p, bool certify) {
     if (p->variant != 0 || p->R > 64 || !p->d_tickets || p->fused == 0) return false;
     if (p->fused > 0) return true;

@@ -1221,7 +1221,12 @@ __device__ __noinline__ bool advance_chain(const FusedArgs &a, uint32_t lane, ui
             }
             const uint32_t mask = __ballot_sync(0xFFFFFFFFu, ready);
             const uint32_t run = mask == 0xFFFFFFFFu ? 32u : (uint32_t)__ffs((int)~mask) - 1u;
-            for (uint32_t i = 0; i < run; ++i) x = mix64(x ^ __shfl_sync(0xFFFFFFFFu, m, i));
+            if (run == 32u) {  // unrolled: the broadcasts are issued ahead of the dependent mix steps
+#pragma unroll
+                for (uint32_t i = 0; i < 32; ++i) x = mix64(x ^ __shfl_sync(0xFFFFFFFFu, m, i));
+            } else {
+                for (uint32_t i = 0; i < run; ++i) x = mix64(x ^ __shfl_sync(0xFFFFFFFFu, m, i));
+            }
             n += run;
             if (run < 32u) break;
         }

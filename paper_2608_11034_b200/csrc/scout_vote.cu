@@ -149,7 +149,10 @@ __global__ void __launch_bounds__(WIDE_THREADS) vote_chunks_wide(
 
 // Certificate: a <- mix64(seed ^ C); a <- mix64(a ^ majority_c) for every chunk
 // in order.  The chain is sequential by construction; one warp streams the
-// hashes in coalesced groups of 32 and lane 0 runs the chain.
+// hashes in coalesced groups of 32 (the next group is in flight while this one
+// is folded) and every lane runs the same chain.  A full group is folded by an
+// unrolled loop, so that the 32 broadcasts are issued ahead of the dependent mix
+// steps instead of one per step.
 __global__ void certificate_chain(uint64_t C, const uint64_t *__restrict__ majority, CertifyOut *out) {
     pdl_wait();
     const uint32_t lane = threadIdx.x;
@@ -159,10 +162,12 @@ __global__ void certificate_chain(uint64_t C, const uint64_t *__restrict__ major
         const uint64_t cur = next;
         const uint64_t nb = base + 32 + lane;
         next = nb < C ? majority[nb] : 0ull;
-        const uint32_t n = (uint32_t)((C - base) < 32 ? (C - base) : 32);
-        for (uint32_t i = 0; i < n; ++i) {
-            const uint64_t hsh = __shfl_sync(0xFFFFFFFFu, cur, i);
-            a = mix64(a ^ hsh);
+        if (C - base >= 32) {
+#pragma unroll
+            for (uint32_t i = 0; i < 32; ++i) a = mix64(a ^ __shfl_sync(0xFFFFFFFFu, cur, i));
+        } else {
+            const uint32_t n = (uint32_t)(C - base);
+            for (uint32_t i = 0; i < n; ++i) a = mix64(a ^ __shfl_sync(0xFFFFFFFFu, cur, i));
         }
     }
     if (lane == 0) {
