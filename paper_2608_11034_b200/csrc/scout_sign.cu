@@ -989,7 +989,16 @@ __global__ void __launch_bounds__(SIGN_THREADS) read_probe(const SignArgs a) {
     const uint64_t warp = (uint64_t)blockIdx.x * (SIGN_THREADS / 32) + (threadIdx.x >> 5);
     const uint64_t n_warps = (uint64_t)gridDim.x * (SIGN_THREADS / 32);
     const uint64_t n_items = a.n_tiles * a.n_replicas;
-    for (uint64_t item = warp; item < n_items; item += n_warps) {
+    // the same work distribution as the scan (see sign_tiles_direct)
+    unsigned long long *work = a.work ? a.work + a.work_parity : nullptr;
+    if (work && warp == 0 && lane == 0) a.work[a.work_parity ^ 1u] = 0ull;
+    const bool dynamic = work != nullptr && n_items > n_warps;
+    uint64_t item = warp;
+    while (item < n_items) {
+        unsigned long long next = 0;
+        if (dynamic) {
+            if (lane == 0) next = atomicAdd(work, 1ull);
+        }
         const uint32_t rr = (uint32_t)(item / a.n_tiles);
         const uint64_t t = a.tile_begin + (item - (uint64_t)rr * a.n_tiles);
         const uint32_t r = a.replica_begin + rr;
@@ -1013,6 +1022,7 @@ __global__ void __launch_bounds__(SIGN_THREADS) read_probe(const SignArgs a) {
 #pragma unroll
         for (int d = 16; d >= 1; d >>= 1) y ^= __shfl_xor_sync(0xFFFFFFFFu, y, d);
         if (lane == 0) a.recs[(uint64_t)r * a.tiles_per_replica + t].h = y;
+        item = dynamic ? n_warps + __shfl_sync(0xFFFFFFFFu, next, 0) : item + n_warps;
     }
 }
 
