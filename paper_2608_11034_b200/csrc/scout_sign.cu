@@ -1384,27 +1384,29 @@ __device__ __forceinline__ void resolve_ticket(const FusedArgs &a, uint32_t lane
 template <int DTSEL>
 __global__ void __launch_bounds__(SIGN_THREADS, SCOUT_MINBLOCKS) certify_tiles(const __grid_constant__ FusedArgs a) {
     const uint32_t lane = threadIdx.x & 31u;
-    const uint64_t warp = (uint64_t)blockIdx.x * (SIGN_THREADS / 32) + (threadIdx.x >> 5);
-    const uint64_t n_warps = (uint64_t)gridDim.x * (SIGN_THREADS / 32);
-    const uint64_t n_items = a.s.n_tiles * a.R;
     // Work items are handed out dynamically (a warp that stops to finalise a chunk simply
     // takes fewer tiles afterwards): every warp starts with item `warp`, later items come
     // from a counter.  The counter of this launch is work[epoch & 1]; the other one is
     // zeroed here for the next launch.  The next item is requested before the current tile
     // is scanned and looked at after it, so the atomic's round trip is never waited for.
-    unsigned long long *work = a.work + (a.epoch & 1u);
-    if (warp == 0 && lane == 0) a.work[(a.epoch & 1u) ^ 1u] = 0ull;
+    // Few values live across the scan of a tile (what can be recomputed from the launch
+    // arguments is): the answers of the two atomics must stay in registers, a spill of
+    // either would wait for its round trip.
+#define N_WARPS ((uint64_t)gridDim.x * (SIGN_THREADS / 32))
+#define N_ITEMS (a.s.n_tiles * a.R)
+    uint64_t item = (uint64_t)blockIdx.x * (SIGN_THREADS / 32) + (threadIdx.x >> 5);
+    if (item == 0 && lane == 0) a.work[(a.epoch & 1u) ^ 1u] = 0ull;
     // the previous tile's ticket: value its atomic returned (lane 0), tiles of its chunk, its chunk
     uint32_t prev_returned = 0, prev_tiles = 0, prev_chunk = 0;
-    const bool more_rounds = n_items > n_warps;  // otherwise every warp has at most its first item
-    uint64_t item = warp;
-    while (item < n_items) {
-        unsigned long long next = n_items;  // "nothing left" unless the counter says otherwise
-        if (more_rounds && lane == 0) next = atomicAdd(work, 1ull);
+    while (item < N_ITEMS) {
+        unsigned long long next = N_ITEMS;  // "nothing left" unless the counter says otherwise
+        if (N_ITEMS > N_WARPS && lane == 0) next = atomicAdd(a.work + (a.epoch & 1u), 1ull);
         const uint64_t t = item / a.R;
         const uint32_t r = (uint32_t)(item - t * a.R);
         const TileDesc td = a.s.tiles[t];
         const uint8_t *tile = a.s.ptrs[(uint64_t)r * a.s.T + td.tensor] + td.off;
+        TileRec *const out = &a.s.recs[(uint64_t)r * a.s.tiles_per_replica + t];
+        uint32_t *const ticket = &a.tickets[a.one_level ? a.C * a.R + td.chunk : (uint64_t)td.chunk * a.R + r];
         // whoever completes this chunk reads its descriptor: have it in L2 by then
         if (lane == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(a.chunks + td.chunk));
         TileRec rec;
@@ -1412,15 +1414,17 @@ __global__ void __launch_bounds__(SIGN_THREADS, SCOUT_MINBLOCKS) certify_tiles(c
         else                      scan_dispatch(td.dtype, tile, td.nbytes, lane, rec);
         if (prev_tiles) resolve_ticket(a, lane, prev_returned, prev_tiles, prev_chunk);
         if (lane == 0) {
-            store_record(&a.s.recs[(uint64_t)r * a.s.tiles_per_replica + t], rec);
+            store_record(out, rec);
             __threadfence();
-            prev_returned = atomicAdd(&a.tickets[a.one_level ? a.C * a.R + td.chunk : (uint64_t)td.chunk * a.R + r], 1u);
+            prev_returned = atomicAdd(ticket, 1u);
         }
         prev_tiles = td.chunk_tiles;
         prev_chunk = td.chunk;
-        item = n_warps + __shfl_sync(0xFFFFFFFFu, next, 0);
+        item = N_WARPS + __shfl_sync(0xFFFFFFFFu, next, 0);
     }
     if (prev_tiles) resolve_ticket(a, lane, prev_returned, prev_tiles, prev_chunk);
+#undef N_WARPS
+#undef N_ITEMS
 }
 
 using FusedKernel = void (*)(const FusedArgs);
