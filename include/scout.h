@@ -279,15 +279,25 @@ SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/)
  *                     3 = read-only probe (measures the memory system only: the
  *                     records it leaves are NOT signatures)
  *   set "fused"       with the default scan (variant 0) and R <= 64 a call can run as
- *                     ONE kernel: the warp that stores the last tile record of a chunk
- *                     finalises it (scout_sign_chunks), and for scout_certify also votes
- *                     it and folds it into the certificate chain; the warp that folds the
- *                     last chunk writes the report block to pinned host memory.
- *                     1: always; 0: never (one kernel per stage: scan, finalise, vote,
- *                     certificate - the form scout_certify_host always uses); -1
- *                     (default): where it measured faster - scout_certify on plans below
- *                     1 GB (latency: one launch instead of four and the copies); larger
- *                     plans and scout_sign_chunks run the stages as separate kernels
+ *                     ONE kernel, in one of two forms.  1 = tickets: the warp that stores
+ *                     the last tile record of a chunk finalises it (scout_sign_chunks), and
+ *                     for scout_certify also votes it and folds it into the certificate
+ *                     chain; the warp that folds the last chunk writes the report block
+ *                     to pinned host memory.  2 = clusters (R <= 8, at most 256 tiles per
+ *                     chunk, else SCOUT_ERR_UNSUPPORTED): a thread-block cluster of R
+ *                     CTAs takes a chunk, CTA r scans replica r's copy and keeps its
+ *                     record in shared memory, the first CTA reads the R hashes through
+ *                     distributed shared memory and votes; chunks of fewer than 16 tiles
+ *                     are taken several at a time.  0 = never (one kernel per stage:
+ *                     scan, finalise, vote, certificate - the form scout_certify_host
+ *                     always uses).  -1 (default) = whichever measured fastest:
+ *                     scout_certify on plans below 1 GiB uses clusters when R <= 8, no
+ *                     chunk has more than 64 tiles and there are at most 1,024 chunks,
+ *                     tickets on other plans up to 16 MiB; larger plans and
+ *                     scout_sign_chunks run the stages as separate kernels
+ *   get "certify_form", "sign_form"  the form (0, 1, 2 as above) scout_certify /
+ *                     scout_sign_chunks would use for this plan now
+ *   get "cluster_ok"  1 if form 2 can run this plan with its current tile size
  *   set "dynamic"     1 (default): the scan's warps take tiles from a work counter as they
  *                     become free; 0: fixed round-robin assignment
  *   set "grid"        CTAs of the scan kernel

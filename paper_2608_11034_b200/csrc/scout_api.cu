@@ -69,9 +69,11 @@ struct scout_plan {
 
     // one-launch path (certify_tiles): per-chunk tickets, launch stamps, chain state
     int fused = -1;               // key "fused": 1 always, 0 never, -1 where it is the faster form (see
-                                  // use_fused); only the default scan (variant 0) has a one-launch form
+                                  // launch_form); only the default scan (variant 0) has a one-launch form
     uint64_t total_bytes = 0;     // R * bytes per replica
     int fused_grid = 0;
+    int cluster_ok = 0;           // the cluster form of the one-launch path can run this plan (upload_tables)
+    uint32_t max_chunk_tiles = 0;
     uint32_t *d_tickets = nullptr, *d_done = nullptr;
     ChainState *d_chain = nullptr;
     unsigned long long *d_work = nullptr;   // one-launch kernels
@@ -231,23 +233,33 @@ int upload_tables(scout_plan *p) {
     SCOUT_CUDA(plan_malloc(p, (void **)&p->d_recs, nt * p->R * sizeof(TileRec)));
     SCOUT_CUDA(cudaMemcpy(p->d_tiles, p->tiles.data(), nt * sizeof(TileDesc), cudaMemcpyHostToDevice));
     SCOUT_CUDA(cudaMemcpy(p->d_chunks, p->chunks.data(), nc * sizeof(ChunkDesc), cudaMemcpyHostToDevice));
-    return SCOUT_OK;
+    p->max_chunk_tiles = 0;
+    for (const ChunkDesc &cd : p->chunks) p->max_chunk_tiles = std::max(p->max_chunk_tiles, cd.ntiles);
+    return cluster_form_possible(p->uniform_dtype, p->R, p->max_chunk_tiles, nc, &p->cluster_ok);
 }
 
-// Is this call made as one launch?  Measured on B200 (key "fused" = -1, the default, follows
-// the measurements; 1 and 0 force either form):
-//   * scout_certify on plans below 1 GB: yes.  One kernel instead of four plus the copies
-//     (12.6 MB: 34 against 42 us on the device, 51 against 67 us per call).
-//   * everything else: no.  With its work handed out dynamically the staged scan reaches
-//     7.2 TB/s on 36 GB of fp32 and 6.25 TB/s on 125 GB of bf16; the one-launch kernel, whose
-//     loop also carries the ticket state (it spills) and takes tiles replica-interleaved, stays
-//     3 to 7 % below that, more than the three small launches it saves.  What the one-launch
-//     form alone offers at large sizes is the certificate chain folded behind the scan (32 ns
-//     per chunk otherwise: 23 us at 717 chunks, 0.8 ms at 24,000).
-bool use_fused(const scout_plan *p, bool certify) {
-    if (p->variant != 0 || p->R > 64 || !p->d_tickets || p->fused == 0) return false;
-    if (p->fused > 0) return true;
-    return certify && p->total_bytes < (1ull << 30);
+// How a call is launched: 0 = one kernel per stage (scan, finalise, vote, certificate chain,
+// linked by programmatic dependent launch), 1 = one kernel with tickets (certify_tiles),
+// 2 = one kernel with a thread-block cluster per chunk (certify_clusters).  Key "fused":
+// 0, 1, 2 force a form (2 only where it can run, else 1); -1, the default, follows what was
+// measured on B200 (device time of scout_certify, L2 flushed between calls):
+//   * scout_certify on a plan below 1 GiB whose chunks have at most 64 tiles and which has
+//     at most 1,024 chunks, R <= 8: clusters.  12.6 MB in 64 KiB chunks: 25 us against 29
+//     (tickets) and 33 (per stage); 50 MB in 256 KiB chunks: 33 against 57 and 46; 201 MB in
+//     1 MiB chunks: 59-68 against 74-84 and 69-73.  With more chunks the sequential
+//     certificate chain (32 ns per chunk) decides and the per-stage form is as fast; with
+//     more tiles per chunk too few CTAs stream (an SM draws about 1/148 of the bandwidth).
+//   * scout_certify on other plans up to 16 MiB: tickets (29-35 us against 33-40).
+//   * everything else: per stage.  With its work handed out dynamically the staged scan
+//     reaches 7.2 TB/s on 36 GB of fp32 and 6.5 TB/s on 125 GB of bf16; the ticket kernel
+//     stays 3 to 9 % below that, more than the three small launches it saves.
+int launch_form(const scout_plan *p, bool certify) {
+    if (p->variant != 0 || p->R > 64 || !p->d_tickets || p->fused == 0) return 0;
+    if (p->fused == 2) return p->cluster_ok ? 2 : 1;
+    if (p->fused == 1) return 1;
+    if (!certify || p->total_bytes >= (1ull << 30)) return 0;
+    if (p->cluster_ok && p->max_chunk_tiles <= 64 && p->chunks.size() <= 1024) return 2;
+    return p->total_bytes <= (16ull << 20) ? 1 : 0;
 }
 
 void fill_sign_launch(const scout_plan *p, SignLaunch &l) {
@@ -293,9 +305,9 @@ int launch_one_kernel(scout_plan *p, cudaStream_t stream, scout_sig_t *d_sigs, b
     f.mode = certify ? 1 : 0;
     f.tickets = p->d_tickets;
     f.work = p->d_work;
-    uint32_t max_tiles = 0;
-    for (const ChunkDesc &cd : p->chunks) max_tiles = std::max(max_tiles, cd.ntiles);
-    f.one_level = (uint64_t)max_tiles * p->R <= 64 ? 1u : 0u;
+    f.one_level = (uint64_t)p->max_chunk_tiles * p->R <= 64 ? 1u : 0u;
+    f.cluster = launch_form(p, certify) == 2 ? 1 : 0;
+    f.max_chunk_tiles = p->max_chunk_tiles;
     if (++p->epoch == 0) p->epoch = 1;  // 0 is the stamp of "never"
     f.epoch = p->epoch;
     if (certify) {
@@ -322,7 +334,7 @@ int launch_one_kernel(scout_plan *p, cudaStream_t stream, scout_sig_t *d_sigs, b
 }
 
 int sign_all(scout_plan *p, cudaStream_t stream, scout_sig_t *d_sigs, CertifyOut *zero_out = nullptr) {
-    if (use_fused(p, false) && !zero_out) return launch_one_kernel(p, stream, d_sigs, false, 0, 0);
+    if (launch_form(p, false) && !zero_out) return launch_one_kernel(p, stream, d_sigs, false, 0, 0);
     SignLaunch l;
     fill_sign_launch(p, l);
     next_work_counter(p, l);
@@ -456,7 +468,7 @@ int vote_and_report(scout_plan *p, cudaStream_t stream, scout_report_t *report,
 int certify_enqueue(scout_plan *p, cudaStream_t stream, uint64_t outlier_cap, uint64_t undecided_cap) {
     int rc = ensure_certify_buffers(p, outlier_cap, undecided_cap);
     if (rc) return rc;
-    if (use_fused(p, true)) {
+    if (launch_form(p, true)) {
         rc = launch_one_kernel(p, stream, p->d_sigs, true, outlier_cap, undecided_cap);
     } else {
         if ((rc = sign_all(p, stream, p->d_sigs, p->d_out))) return rc;
@@ -882,7 +894,8 @@ int scout_plan_set(scout_plan_t *p, const char *key, int64_t value) {
         return SCOUT_OK;
     }
     if (!std::strcmp(key, "fused")) {
-        if (value < -1 || value > 1) return SCOUT_ERR_INVALID;
+        if (value < -1 || value > 2) return SCOUT_ERR_INVALID;
+        if (value == 2 && !p->cluster_ok) return SCOUT_ERR_UNSUPPORTED;
         p->fused = (int)value;
         return SCOUT_OK;
     }
@@ -930,9 +943,12 @@ int scout_plan_get(const scout_plan_t *p, const char *key, int64_t *value) {
         return guards_intact(p, value);
     }
     else if (!std::strcmp(key, "fused")) *value = p->fused;
+    else if (!std::strcmp(key, "certify_form")) *value = launch_form(p, true);
+    else if (!std::strcmp(key, "sign_form")) *value = launch_form(p, false);
+    else if (!std::strcmp(key, "cluster_ok")) *value = p->cluster_ok;
     else if (!std::strcmp(key, "dynamic")) *value = p->dynamic;
-    else if (!std::strcmp(key, "sign_kernels")) *value = use_fused(p, false) ? 1 : 2;    // scan, finalise
-    else if (!std::strcmp(key, "certify_kernels")) *value = use_fused(p, true) ? 1 : 4;  // + vote, certificate chain
+    else if (!std::strcmp(key, "sign_kernels")) *value = launch_form(p, false) ? 1 : 2;    // scan, finalise
+    else if (!std::strcmp(key, "certify_kernels")) *value = launch_form(p, true) ? 1 : 4;  // + vote, certificate chain
     else if (!std::strcmp(key, "last_sign_ns")) {
         // device time of the most recent scan kernel; the stream must have been synchronised
         if (!p->timing || p->timed_launches == 0) return SCOUT_ERR_INVALID;

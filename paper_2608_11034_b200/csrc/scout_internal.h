@@ -207,9 +207,12 @@ struct FusedLaunch {
     uint32_t one_level;         // 1: every chunk has at most 64 (tile, replica) items: chunk tickets only
     ChainState *chain;          // mode 1: zero on entry; left zero on exit
     CertifyHost *host;          // mode 1: pinned host memory (device-accessible address)
+    int cluster;                // 1: one thread-block cluster per chunk (certify_clusters) instead of tickets
+    uint32_t max_chunk_tiles;   // most tiles any chunk has
 };
 int launch_fused(const FusedLaunch &l, cudaStream_t stream);
 int fused_grid_size(int uniform_dtype, int device, int *grid);
+int cluster_form_possible(int uniform_dtype, uint32_t R, uint32_t max_tiles, uint64_t C, int *ok);
 int sign_grid_size(int variant, int uniform_dtype, int device, int *grid);
 int launch_bounded_wait_selftest(uint64_t limit_ns, uint64_t *d_out, cudaStream_t stream);
 

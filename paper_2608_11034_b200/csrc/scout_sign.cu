@@ -1066,6 +1066,8 @@ __device__ __forceinline__ uint64_t combine_weight(uint32_t nt, uint64_t nbytes,
     return pow_p(rows_last + (uint64_t)tile_rows * (n_full - 1 - last_t));
 }
 
+// SHARED: the records sit in this CTA's shared memory (plain loads) instead of global memory.
+template <bool SHARED = false>
 __device__ __forceinline__ scout_sig_t combine_tiles(const TileRec *tr, uint32_t nt, uint64_t nbytes,
                                                      uint64_t k, uint32_t dtype, uint64_t meta,
                                                      uint64_t p_stride, uint64_t weight, uint32_t lane) {
@@ -1074,7 +1076,7 @@ __device__ __forceinline__ scout_sig_t combine_tiles(const TileRec *tr, uint32_t
     uint32_t nan_count = 0, inf_count = 0;
     const uint32_t n_full = nt - 1;
     for (uint32_t t = lane; t < n_full; t += 32) {
-        const TileRec x = load_record(tr + t);
+        const TileRec x = SHARED ? tr[t] : load_record(tr + t);
         h = h * p_stride + x.h;
         s += x.sum;
         q += x.sumsq;
@@ -1083,7 +1085,7 @@ __device__ __forceinline__ scout_sig_t combine_tiles(const TileRec *tr, uint32_t
     }
     if (lane < n_full) h *= weight;
     if (lane == (n_full & 31u)) {  // the last (possibly short) tile: nothing follows it
-        const TileRec x = load_record(tr + n_full);
+        const TileRec x = SHARED ? tr[n_full] : load_record(tr + n_full);
         h += x.h;
         s += x.sum;
         q += x.sumsq;
@@ -1196,6 +1198,7 @@ struct FusedArgs {
     CertifyHost *host;
     unsigned long long *work;  // two work counters, used alternately by successive launches
     uint32_t one_level;        // tickets: chunk counters only (chunks with few items)
+    uint32_t cluster_batch;    // certify_clusters: chunks a cluster takes at once
 };
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
@@ -1285,10 +1288,13 @@ __device__ __noinline__ void publish_report(const FusedArgs &a, uint32_t lane, u
         *reinterpret_cast<volatile uint32_t *>(&a.host->dev_err) = a.s.error ? __ldcg(a.s.error) : 0u;
         *(volatile uint64_t *)&a.chain->next = 0ull;
         *(volatile uint64_t *)&a.chain->a = 0ull;
-        __threadfence_system();
+        __threadfence();   // the host reads the report after the stream has completed: no system fence needed
         atomicExch(&a.chain->lock, 0u);
     }
 }
+
+__device__ __noinline__ void chunk_vote_and_fold(const FusedArgs &a, uint32_t c, uint64_t e0, uint64_t e1,
+                                                 uint32_t lane);
 
 // The last tile record of chunk c has been stored: finalise, vote, fold.
 __device__ __noinline__ void chunk_complete(const FusedArgs &a, uint32_t c, uint32_t lane) {
@@ -1328,6 +1334,13 @@ __device__ __noinline__ void chunk_complete(const FusedArgs &a, uint32_t c, uint
     // both ticket levels of this chunk go back to zero for the next launch
     for (uint32_t r = lane; r <= a.R; r += 32) a.tickets[r < a.R ? (uint64_t)c * a.R + r : a.C * a.R + c] = 0u;
     if (a.mode == 0) return;
+    chunk_vote_and_fold(a, c, e0, e1, lane);
+}
+
+// The R records of chunk c exist and lane j holds the hashes of replicas j and j + 32:
+// vote the chunk, count it, and fold the certificate chain as far as it can be folded.
+__device__ __noinline__ void chunk_vote_and_fold(const FusedArgs &a, uint32_t c, uint64_t e0, uint64_t e1,
+                                                 uint32_t lane) {
     uint64_t bitmap, majority;
     const uint32_t st = vote_chunk(a.R, c, e0, e1, lane, a.v, bitmap, majority);
     if (a.C <= SMALL_CHAIN) {
@@ -1427,7 +1440,97 @@ __global__ void __launch_bounds__(SIGN_THREADS, SCOUT_MINBLOCKS) certify_tiles(c
 #undef N_ITEMS
 }
 
+// ---- one launch, one thread-block cluster per chunk -----------------------------------
+// certify_clusters: the same path for plans made of many small chunks.  A cluster of R
+// CTAs takes chunk c; CTA r of it scans replica r's copy of the chunk (one warp per tile,
+// the tile geometry of the plan, records into shared memory), combines them after a
+// CTA barrier and keeps the finished record in shared memory.  After a cluster barrier
+// the first CTA reads the R hashes out of the other CTAs' shared memory and votes.  No
+// tile record, ticket or fence goes through global memory on the way to the vote: from
+// the arrival of a chunk's last byte to its vote there are two barriers and no L2 round
+// trip.  Only the job-wide steps (counters, certificate chain, report) use global
+// atomics, once per chunk.  The tile table is not read: a chunk's tiles follow from its
+// descriptor.
+constexpr int CLUSTER_THREADS = 512;
+constexpr uint32_t CLUSTER_MAX_TILES = 256;   // records of one (chunk, replica) held in shared memory
+constexpr uint32_t CLUSTER_MAX_R = 8;         // portable cluster size
+
+__device__ __forceinline__ uint32_t cluster_cta_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// A 64-bit value at the same shared-memory address in CTA `rank` of this cluster.
+__device__ __forceinline__ uint64_t ld_cluster_u64(const void *local, uint32_t rank) {
+    uint32_t remote;
+    uint64_t v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local)), "r"(rank));
+    asm volatile("ld.shared::cluster.u64 %0, [%1];" : "=l"(v) : "r"(remote) : "memory");
+    return v;
+}
+
+template <int DTSEL>
+__global__ void __launch_bounds__(CLUSTER_THREADS, 2) certify_clusters(const __grid_constant__ FusedArgs a) {
+    constexpr uint32_t WARPS = CLUSTER_THREADS / 32;
+    __shared__ TileRec s_rec[CLUSTER_MAX_TILES];
+    __shared__ __align__(16) scout_sig_t s_sig[WARPS];
+    __shared__ ChunkDesc s_chunk[WARPS];
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const uint32_t r = cluster_cta_rank();            // cluster dimension = R
+    // A cluster takes `batch` consecutive chunks at once (a power of two; more than one only
+    // when every chunk has at most WARPS / batch tiles): warps_per_chunk warps scan a chunk.
+    const uint32_t batch = a.cluster_batch, warps_per_chunk = WARPS / batch;
+    const uint64_t c_first = (uint64_t)(blockIdx.x / a.R) * batch;
+    const uint32_t tile_bytes = a.tile_rows * ROW_BYTES;
+    {
+        const uint32_t b = warp / warps_per_chunk, j0 = warp - b * warps_per_chunk;
+        const uint64_t c = c_first + b;
+        if (c < a.C) {
+            const ChunkDesc cd = a.chunks[c];
+            if (j0 == 0 && lane == 0) s_chunk[b] = cd;
+            const uint8_t *base = a.s.ptrs[(uint64_t)r * a.s.T + cd.tensor] + cd.byte_offset;
+            TileRec *recs = s_rec + (batch > 1 ? b * warps_per_chunk : 0u);
+            for (uint32_t j = j0; j < cd.ntiles; j += warps_per_chunk) {
+                const uint64_t off = (uint64_t)j * tile_bytes;
+                const uint32_t nbytes = (uint32_t)min((uint64_t)tile_bytes, cd.nbytes - off);
+                TileRec rec;
+                if constexpr (DTSEL >= 0) scan_tile<DTSEL>(base + off, nbytes, lane, rec);
+                else                      scan_dispatch(cd.dtype, base + off, nbytes, lane, rec);
+                if (lane == 0) recs[j] = rec;
+            }
+        }
+    }
+    __syncthreads();
+    const uint64_t c = c_first + warp;                // from here on warp b works on chunk b of the batch
+    const bool mine = warp < batch && c < a.C;
+    if (mine) {
+        const ChunkDesc cd = s_chunk[warp];
+        const scout_sig_t o = combine_tiles<true>(s_rec + (batch > 1 ? warp * warps_per_chunk : 0u), cd.ntiles,
+                                                  cd.nbytes, cd.k, cd.dtype, cd.meta, a.p_stride,
+                                                  combine_weight(cd.ntiles, cd.nbytes, a.tile_rows, lane), lane);
+        if (lane == 0) {
+            a.sigs[c * a.R + r] = o;
+            s_sig[warp] = o;
+        }
+    }
+    if (a.mode == 0) return;
+    cluster_barrier();   // every CTA of the cluster has its records in shared memory
+    uint64_t e0 = 0;
+    if (r == 0 && mine && lane < a.R) e0 = ld_cluster_u64(&s_sig[warp].hash, lane);
+    cluster_barrier();   // nobody leaves while its shared memory may still be read
+    if (r == 0 && mine) chunk_vote_and_fold(a, (uint32_t)c, e0, 0ull, lane);
+}
+
 using FusedKernel = void (*)(const FusedArgs);
+FusedKernel cluster_kernel(int uniform) {
+    if (uniform == SCOUT_DT_F32) return certify_clusters<SCOUT_DT_F32>;
+    if (uniform == SCOUT_DT_BF16) return certify_clusters<SCOUT_DT_BF16>;
+    return certify_clusters<-1>;
+}
+
 FusedKernel fused_kernel(int uniform) {
     if (uniform == SCOUT_DT_F32) return certify_tiles<SCOUT_DT_F32>;
     if (uniform == SCOUT_DT_BF16) return certify_tiles<SCOUT_DT_BF16>;
@@ -1442,6 +1545,30 @@ int fused_grid_size(int uniform_dtype, int device, int *grid) {
     SCOUT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_kernel(uniform_dtype), SIGN_THREADS, 0));
     if (per_sm < 1) per_sm = 1;
     *grid = sms * per_sm;
+    return SCOUT_OK;
+}
+
+// Whether the cluster form can run a plan of R replicas whose chunks have at most max_tiles
+// tiles on this device: R CTAs of CLUSTER_THREADS threads must fit one cluster.
+int cluster_form_possible(int uniform_dtype, uint32_t R, uint32_t max_tiles, uint64_t C, int *ok) {
+    *ok = 0;
+    if (R < 1 || R > CLUSTER_MAX_R || max_tiles > CLUSTER_MAX_TILES || C * R > 0x7FFFFFFFull || C == 0) return SCOUT_OK;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(R);
+    cfg.blockDim = dim3(CLUSTER_THREADS);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = R;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, cluster_kernel(uniform_dtype), &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        return SCOUT_OK;
+    }
+    *ok = n > 0;
     return SCOUT_OK;
 }
 
@@ -1478,6 +1605,26 @@ int launch_fused(const FusedLaunch &l, cudaStream_t stream) {
     a.host = l.host;
     a.work = l.work;
     a.one_level = l.one_level;
+    a.cluster_batch = 1;
+    if (l.cluster) {
+        // chunks with few tiles are taken several at a time, so that every warp of a CTA has a tile
+        uint32_t batch = 1;
+        while (batch < CLUSTER_THREADS / 32 && 2 * batch * l.max_chunk_tiles <= CLUSTER_THREADS / 32) batch *= 2;
+        a.cluster_batch = batch;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(((l.C + batch - 1) / batch) * l.R));
+        cfg.blockDim = dim3(CLUSTER_THREADS);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = l.R;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        SCOUT_CUDA(cudaLaunchKernelEx(&cfg, cluster_kernel(l.sign.uniform_dtype), a));
+        return SCOUT_OK;
+    }
     const uint64_t items = l.sign.n_tiles * l.R;
     const uint64_t want = (items + SIGN_THREADS / 32 - 1) / (SIGN_THREADS / 32);
     int grid = l.sign.grid;

@@ -22,7 +22,7 @@ def _binding():
 
 # direct loads with one kernel per stage, the same scan with the whole call as one launch, register
 # prefetch, per-warp bulk-async ring, block-wide ring
-VARIANTS = ["unfused", "fused", 1, 2, 4]
+VARIANTS = ["unfused", "fused", "cluster", 1, 2, 4]
 
 
 def _compare_everything(w, views, chunk_bytes=None, tile_bytes=None, variant=None):
@@ -68,7 +68,7 @@ def _odd_workload(dtype, seed):
 
 
 @pytest.mark.parametrize("dtype", ["u8", "f32", "bf16", "i64", "f16", "f64", "i32"])
-@pytest.mark.parametrize("tile_bytes,variant", [(2048, "fused"), (4096, "fused"), (2048, "unfused"), (4096, "unfused"),
+@pytest.mark.parametrize("tile_bytes,variant", [(2048, "fused"), (4096, "fused"), (2048, "cluster"), (4096, "cluster"), (2048, "unfused"), (4096, "unfused"),
                                                 (4096, 1), (8192, 1),
                                                 (4096, 2), (8192, 2), (32768, 2), (4096, 4), (8192, 4), (32768, 4)])
 def test_every_dtype_and_ragged_sizes(dtype, tile_bytes, variant):
