@@ -74,6 +74,7 @@ struct scout_plan {
     int fused_grid = 0;
     int cluster_ok = 0;           // the cluster form of the one-launch path can run this plan (upload_tables)
     uint32_t max_chunk_tiles = 0;
+    uint32_t cluster_batch = 1, cluster_split = 1;   // geometry of the cluster form (cluster_form_possible)
     uint32_t *d_tickets = nullptr, *d_done = nullptr;
     ChainState *d_chain = nullptr;
     unsigned long long *d_work = nullptr;   // one-launch kernels
@@ -235,7 +236,8 @@ int upload_tables(scout_plan *p) {
     SCOUT_CUDA(cudaMemcpy(p->d_chunks, p->chunks.data(), nc * sizeof(ChunkDesc), cudaMemcpyHostToDevice));
     p->max_chunk_tiles = 0;
     for (const ChunkDesc &cd : p->chunks) p->max_chunk_tiles = std::max(p->max_chunk_tiles, cd.ntiles);
-    return cluster_form_possible(p->uniform_dtype, p->R, p->max_chunk_tiles, nc, &p->cluster_ok);
+    return cluster_form_possible(p->uniform_dtype, p->R, p->max_chunk_tiles, nc, &p->cluster_ok,
+                                 &p->cluster_batch, &p->cluster_split);
 }
 
 // How a call is launched: 0 = one kernel per stage (scan, finalise, vote, certificate chain,
@@ -258,7 +260,7 @@ int launch_form(const scout_plan *p, bool certify) {
     if (p->fused == 2) return p->cluster_ok ? 2 : 1;
     if (p->fused == 1) return 1;
     if (!certify || p->total_bytes >= (1ull << 30)) return 0;
-    if (p->cluster_ok && p->max_chunk_tiles <= 64 && p->chunks.size() <= 1024) return 2;
+    if (p->cluster_ok && p->max_chunk_tiles <= 64 * p->cluster_split && p->chunks.size() <= 1024) return 2;
     return p->total_bytes <= (16ull << 20) ? 1 : 0;
 }
 
@@ -307,7 +309,8 @@ int launch_one_kernel(scout_plan *p, cudaStream_t stream, scout_sig_t *d_sigs, b
     f.work = p->d_work;
     f.one_level = (uint64_t)p->max_chunk_tiles * p->R <= 64 ? 1u : 0u;
     f.cluster = launch_form(p, certify) == 2 ? 1 : 0;
-    f.max_chunk_tiles = p->max_chunk_tiles;
+    f.cluster_batch = p->cluster_batch;
+    f.cluster_split = p->cluster_split;
     if (++p->epoch == 0) p->epoch = 1;  // 0 is the stamp of "never"
     f.epoch = p->epoch;
     if (certify) {

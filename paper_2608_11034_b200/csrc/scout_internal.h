@@ -208,11 +208,13 @@ struct FusedLaunch {
     ChainState *chain;          // mode 1: zero on entry; left zero on exit
     CertifyHost *host;          // mode 1: pinned host memory (device-accessible address)
     int cluster;                // 1: one thread-block cluster per chunk (certify_clusters) instead of tickets
-    uint32_t max_chunk_tiles;   // most tiles any chunk has
+    uint32_t cluster_batch;     // cluster form: chunks a cluster takes at once (cluster_form_possible)
+    uint32_t cluster_split;     // cluster form: CTAs per replica of a chunk
 };
 int launch_fused(const FusedLaunch &l, cudaStream_t stream);
 int fused_grid_size(int uniform_dtype, int device, int *grid);
-int cluster_form_possible(int uniform_dtype, uint32_t R, uint32_t max_tiles, uint64_t C, int *ok);
+int cluster_form_possible(int uniform_dtype, uint32_t R, uint32_t max_tiles, uint64_t C, int *ok,
+                          uint32_t *batch, uint32_t *split);
 int sign_grid_size(int variant, int uniform_dtype, int device, int *grid);
 int launch_bounded_wait_selftest(uint64_t limit_ns, uint64_t *d_out, cudaStream_t stream);
 

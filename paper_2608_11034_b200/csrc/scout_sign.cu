@@ -1199,6 +1199,7 @@ struct FusedArgs {
     unsigned long long *work;  // two work counters, used alternately by successive launches
     uint32_t one_level;        // tickets: chunk counters only (chunks with few items)
     uint32_t cluster_batch;    // certify_clusters: chunks a cluster takes at once
+    uint32_t cluster_split;    // certify_clusters: CTAs that share one replica's copy of a chunk
 };
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
@@ -1441,87 +1442,115 @@ __global__ void __launch_bounds__(SIGN_THREADS, SCOUT_MINBLOCKS) certify_tiles(c
 }
 
 // ---- one launch, one thread-block cluster per chunk -----------------------------------
-// certify_clusters: the same path for plans made of many small chunks.  A cluster of R
-// CTAs takes chunk c; CTA r of it scans replica r's copy of the chunk (one warp per tile,
-// the tile geometry of the plan, records into shared memory), combines them after a
-// CTA barrier and keeps the finished record in shared memory.  After a cluster barrier
-// the first CTA reads the R hashes out of the other CTAs' shared memory and votes.  No
-// tile record, ticket or fence goes through global memory on the way to the vote: from
-// the arrival of a chunk's last byte to its vote there are two barriers and no L2 round
-// trip.  Only the job-wide steps (counters, certificate chain, report) use global
-// atomics, once per chunk.  The tile table is not read: a chunk's tiles follow from its
-// descriptor.
+// certify_clusters: the same path for plans made of many small chunks.  A cluster of
+// R * split CTAs takes chunk c; `split` CTAs share replica r's copy of the chunk (one warp
+// per tile, the tile geometry of the plan).  Tile records are stored straight into the
+// shared memory of the replica's first CTA, which combines them after a barrier and
+// stores the finished hash into the shared memory of the cluster's first CTA; that one
+// votes after a second barrier.  No tile record, ticket or fence goes through global
+// memory on the way to the vote: from the arrival of a chunk's last byte to its vote
+// there are two barriers and no L2 round trip.  Only the job-wide steps (counters,
+// certificate chain, report) use global atomics, once per chunk.  The tile table is not
+// read: a chunk's tiles follow from its descriptor.  Chunks of fewer than 16 tiles are
+// taken `batch` at a time, so that every warp of a CTA has a tile.
 constexpr int CLUSTER_THREADS = 512;
-constexpr uint32_t CLUSTER_MAX_TILES = 256;   // records of one (chunk, replica) held in shared memory
-constexpr uint32_t CLUSTER_MAX_R = 8;         // portable cluster size
+constexpr uint32_t CLUSTER_MAX_TILES = 512;   // records of one (chunk, replica) held in shared memory
+constexpr uint32_t CLUSTER_MAX_CTAS = 8;      // portable cluster size: R * split
 
 __device__ __forceinline__ uint32_t cluster_cta_rank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
     return r;
 }
-__device__ __forceinline__ void cluster_barrier() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+__device__ __forceinline__ void cluster_arrive() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
 }
-// A 64-bit value at the same shared-memory address in CTA `rank` of this cluster.
-__device__ __forceinline__ uint64_t ld_cluster_u64(const void *local, uint32_t rank) {
+__device__ __forceinline__ void cluster_wait() {
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// The address of `local` (a shared-memory object of this CTA) in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t cluster_address(const void *local, uint32_t rank) {
     uint32_t remote;
-    uint64_t v;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local)), "r"(rank));
-    asm volatile("ld.shared::cluster.u64 %0, [%1];" : "=l"(v) : "r"(remote) : "memory");
-    return v;
+    return remote;
+}
+__device__ __forceinline__ void st_cluster_u64(uint32_t addr, uint64_t v) {
+    asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(addr), "l"(v) : "memory");
+}
+__device__ __forceinline__ void st_cluster_record(uint32_t addr, const TileRec &rec) {
+    asm volatile("st.shared::cluster.v2.u64 [%0], {%1, %2};" ::"r"(addr), "l"(rec.h),
+                 "l"((uint64_t)__double_as_longlong(rec.sum)) : "memory");
+    asm volatile("st.shared::cluster.v2.u64 [%0], {%1, %2};" ::"r"(addr + 16u),
+                 "l"((uint64_t)__double_as_longlong(rec.sumsq)),
+                 "l"((uint64_t)rec.nan_count | ((uint64_t)rec.inf_count << 32)) : "memory");
 }
 
 template <int DTSEL>
 __global__ void __launch_bounds__(CLUSTER_THREADS, 2) certify_clusters(const __grid_constant__ FusedArgs a) {
     constexpr uint32_t WARPS = CLUSTER_THREADS / 32;
-    __shared__ TileRec s_rec[CLUSTER_MAX_TILES];
-    __shared__ __align__(16) scout_sig_t s_sig[WARPS];
+    __shared__ __align__(16) TileRec s_rec[CLUSTER_MAX_TILES];
+    __shared__ uint64_t s_hash[WARPS][CLUSTER_MAX_CTAS];   // first CTA: hash of (chunk of the batch, replica)
     __shared__ ChunkDesc s_chunk[WARPS];
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    const uint32_t r = cluster_cta_rank();            // cluster dimension = R
-    // A cluster takes `batch` consecutive chunks at once (a power of two; more than one only
-    // when every chunk has at most WARPS / batch tiles): warps_per_chunk warps scan a chunk.
-    const uint32_t batch = a.cluster_batch, warps_per_chunk = WARPS / batch;
-    const uint64_t c_first = (uint64_t)(blockIdx.x / a.R) * batch;
+    const uint32_t split = a.cluster_split, batch = a.cluster_batch;
+    const uint32_t rank = cluster_cta_rank();         // cluster dimension = R * split
+    const uint32_t r = rank / split, part = rank - r * split;
+    const bool remote = split > 1 || a.mode != 0;     // does anything cross CTAs in this launch?
+    // Stores into another CTA's shared memory need that CTA to have started: arrive now,
+    // wait when the first loads are on their way.
+    if (remote) cluster_arrive();
+    const uint32_t warps_per_chunk = WARPS / batch;   // batch > 1 only with split == 1
+    const uint64_t c_first = (uint64_t)(blockIdx.x / (a.R * split)) * batch;
     const uint32_t tile_bytes = a.tile_rows * ROW_BYTES;
-    {
-        const uint32_t b = warp / warps_per_chunk, j0 = warp - b * warps_per_chunk;
-        const uint64_t c = c_first + b;
-        if (c < a.C) {
-            const ChunkDesc cd = a.chunks[c];
-            if (j0 == 0 && lane == 0) s_chunk[b] = cd;
-            const uint8_t *base = a.s.ptrs[(uint64_t)r * a.s.T + cd.tensor] + cd.byte_offset;
-            TileRec *recs = s_rec + (batch > 1 ? b * warps_per_chunk : 0u);
-            for (uint32_t j = j0; j < cd.ntiles; j += warps_per_chunk) {
-                const uint64_t off = (uint64_t)j * tile_bytes;
-                const uint32_t nbytes = (uint32_t)min((uint64_t)tile_bytes, cd.nbytes - off);
-                TileRec rec;
-                if constexpr (DTSEL >= 0) scan_tile<DTSEL>(base + off, nbytes, lane, rec);
-                else                      scan_dispatch(cd.dtype, base + off, nbytes, lane, rec);
-                if (lane == 0) recs[j] = rec;
+    const uint32_t b = warp / warps_per_chunk, j0 = warp - b * warps_per_chunk;
+    const uint64_t c_scan = c_first + b;
+    ChunkDesc cd;
+    cd.ntiles = 0;
+    const uint8_t *base = nullptr;
+    if (c_scan < a.C) {
+        cd = a.chunks[c_scan];
+        base = a.s.ptrs[(uint64_t)r * a.s.T + cd.tensor] + cd.byte_offset;
+    }
+    if (remote) cluster_wait();
+    if (c_scan < a.C) {
+        if (part == 0 && j0 == 0 && lane == 0) s_chunk[b] = cd;
+        const uint32_t slot0 = batch > 1 ? b * warps_per_chunk : 0u;
+        const uint32_t home = split > 1 ? cluster_address(s_rec, r * split) : 0u;
+        for (uint32_t j = part * warps_per_chunk + j0; j < cd.ntiles; j += split * warps_per_chunk) {
+            const uint64_t off = (uint64_t)j * tile_bytes;
+            const uint32_t nbytes = (uint32_t)min((uint64_t)tile_bytes, cd.nbytes - off);
+            TileRec rec;
+            if constexpr (DTSEL >= 0) scan_tile<DTSEL>(base + off, nbytes, lane, rec);
+            else                      scan_dispatch(cd.dtype, base + off, nbytes, lane, rec);
+            if (lane == 0) {
+                if (split > 1) st_cluster_record(home + (slot0 + j) * (uint32_t)sizeof(TileRec), rec);
+                else           s_rec[slot0 + j] = rec;
             }
         }
     }
-    __syncthreads();
+    // every record of (chunk, replica r) is in the shared memory of the replica's first CTA
+    if (split > 1) {
+        cluster_arrive();
+        cluster_wait();
+    } else {
+        __syncthreads();
+    }
     const uint64_t c = c_first + warp;                // from here on warp b works on chunk b of the batch
     const bool mine = warp < batch && c < a.C;
-    if (mine) {
-        const ChunkDesc cd = s_chunk[warp];
-        const scout_sig_t o = combine_tiles<true>(s_rec + (batch > 1 ? warp * warps_per_chunk : 0u), cd.ntiles,
-                                                  cd.nbytes, cd.k, cd.dtype, cd.meta, a.p_stride,
-                                                  combine_weight(cd.ntiles, cd.nbytes, a.tile_rows, lane), lane);
+    if (mine && part == 0) {
+        const ChunkDesc my = s_chunk[warp];
+        const scout_sig_t o = combine_tiles<true>(s_rec + (batch > 1 ? warp * warps_per_chunk : 0u), my.ntiles,
+                                                  my.nbytes, my.k, my.dtype, my.meta, a.p_stride,
+                                                  combine_weight(my.ntiles, my.nbytes, a.tile_rows, lane), lane);
         if (lane == 0) {
             a.sigs[c * a.R + r] = o;
-            s_sig[warp] = o;
+            if (a.mode != 0) st_cluster_u64(cluster_address(&s_hash[warp][r], 0), o.hash);
         }
     }
     if (a.mode == 0) return;
-    cluster_barrier();   // every CTA of the cluster has its records in shared memory
-    uint64_t e0 = 0;
-    if (r == 0 && mine && lane < a.R) e0 = ld_cluster_u64(&s_sig[warp].hash, lane);
-    cluster_barrier();   // nobody leaves while its shared memory may still be read
-    if (r == 0 && mine) chunk_vote_and_fold(a, (uint32_t)c, e0, 0ull, lane);
+    cluster_arrive();
+    cluster_wait();      // the R hashes of every chunk of the batch are in the first CTA
+    if (rank == 0 && mine) chunk_vote_and_fold(a, (uint32_t)c, lane < a.R ? s_hash[warp][lane] : 0ull, 0ull, lane);
 }
 
 using FusedKernel = void (*)(const FusedArgs);
@@ -1549,16 +1578,38 @@ int fused_grid_size(int uniform_dtype, int device, int *grid) {
 }
 
 // Whether the cluster form can run a plan of R replicas whose chunks have at most max_tiles
-// tiles on this device: R CTAs of CLUSTER_THREADS threads must fit one cluster.
-int cluster_form_possible(int uniform_dtype, uint32_t R, uint32_t max_tiles, uint64_t C, int *ok) {
+// tiles on this device, and with which geometry.  Chunks with few tiles are taken `batch`
+// at a time, so that every warp of a CTA has a tile; chunks with many tiles are shared by
+// `split` CTAs per replica while the cluster stays within its size, every CTA keeps at
+// least a tile per warp ...
+int cluster_form_possible(int uniform_dtype, uint32_t R, uint32_t max_tiles, uint64_t C, int *ok,
+                          uint32_t *batch_out, uint32_t *split_out) {
     *ok = 0;
-    if (R < 1 || R > CLUSTER_MAX_R || max_tiles > CLUSTER_MAX_TILES || C * R > 0x7FFFFFFFull || C == 0) return SCOUT_OK;
+    constexpr uint32_t WARPS = CLUSTER_THREADS / 32;
+    uint32_t batch = 1, split = 1;
+    while (batch < WARPS && 2 * batch * max_tiles <= WARPS) batch *= 2;
+    // ... and only while all CTAs of the launch are resident at once (two per SM): a second
+    // wave of CTAs costs more than the finer split gains (measured: 201 MB in 1 MiB chunks,
+    // R = 3, 59 us with 201 CTAs, 68 us with 402)
+    int device = 0, sms = 0;
+    SCOUT_CUDA(cudaGetDevice(&device));
+    SCOUT_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+    const uint64_t clusters = (C + batch - 1) / batch;
+    while (2 * split * R <= CLUSTER_MAX_CTAS && max_tiles >= 2 * split * WARPS &&
+           clusters * R * 2 * split <= 2ull * (uint64_t)sms)
+        split *= 2;
+    *batch_out = batch;
+    *split_out = split;
+    if (R < 1 || R > CLUSTER_MAX_CTAS || max_tiles > CLUSTER_MAX_TILES || C * CLUSTER_MAX_CTAS > 0x7FFFFFFFull || C == 0)
+        return SCOUT_OK;
+    uint32_t ctas = R;                     // the largest cluster launch_fused may ask for
+    while (2 * ctas <= CLUSTER_MAX_CTAS) ctas *= 2;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(R);
+    cfg.gridDim = dim3(ctas);
     cfg.blockDim = dim3(CLUSTER_THREADS);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = R;
+    attr[0].val.clusterDim.x = ctas;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
@@ -1606,18 +1657,18 @@ int launch_fused(const FusedLaunch &l, cudaStream_t stream) {
     a.work = l.work;
     a.one_level = l.one_level;
     a.cluster_batch = 1;
+    a.cluster_split = 1;
     if (l.cluster) {
-        // chunks with few tiles are taken several at a time, so that every warp of a CTA has a tile
-        uint32_t batch = 1;
-        while (batch < CLUSTER_THREADS / 32 && 2 * batch * l.max_chunk_tiles <= CLUSTER_THREADS / 32) batch *= 2;
+        const uint32_t batch = l.cluster_batch, split = l.cluster_split;
         a.cluster_batch = batch;
+        a.cluster_split = split;
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)(((l.C + batch - 1) / batch) * l.R));
+        cfg.gridDim = dim3((unsigned)(((l.C + batch - 1) / batch) * l.R * split));
         cfg.blockDim = dim3(CLUSTER_THREADS);
         cfg.stream = stream;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = l.R;
+        attr[0].val.clusterDim.x = l.R * split;
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;

@@ -73,11 +73,11 @@ def gpu_plan(w, chunk_bytes=None, tags=None, tile_bytes=None, variant=None):
         binding.scout_plan_set(plan.handle, "fused", 0)
     elif variant == "fused":      # the default scan, the whole call as one launch (tickets)
         binding.scout_plan_set(plan.handle, "fused", 1)
-    elif variant == "cluster":    # one launch, a thread-block cluster per chunk (R <= 8, <= 256 tiles per chunk)
+    elif variant == "cluster":    # one launch, a thread-block cluster per chunk (R <= 8, <= 512 tiles per chunk)
         import pytest
         if not binding.scout_plan_get(plan.handle, "cluster_ok"):
             plan.close()
-            pytest.skip("the cluster form does not fit this plan (R > 8 or more than 256 tiles per chunk)")
+            pytest.skip("the cluster form does not fit this plan (R > 8 or more than 512 tiles per chunk)")
         binding.scout_plan_set(plan.handle, "fused", 2)
     elif variant is not None:
         binding.scout_plan_set(plan.handle, "variant", variant)

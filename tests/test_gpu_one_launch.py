@@ -186,9 +186,9 @@ def test_cluster_form_with_one_to_eight_replicas_and_the_limits():
                 assert got["outliers"] == want["outliers"] and got["undecided"] == want["undecided"]
         helpers.assert_guards(plan)
         plan.close()
-    # nine replicas, or more than 256 tiles in a chunk: the form is refused, the others still run
+    # nine replicas, or more than 512 tiles in a chunk: the form is refused, the others still run
     spec = inputs.TensorSpec("x", (1 << 20,), "f32", "normal", 1.0)
-    for R, chunk_bytes, tile in ((9, 65536, None), (3, 1 << 20, 2048)):
+    for R, chunk_bytes, tile in ((9, 65536, None), (3, 2 << 20, 2048)):
         w = inputs.Workload("no", 0, "x", R, chunk_bytes, [spec], 3)
         plan = helpers.gpu_plan(w, tile_bytes=tile)
         assert B.scout_plan_get(plan.handle, "cluster_ok") == 0
