@@ -89,6 +89,10 @@ def parse_args():
     ap.add_argument("--variant", type=int, default=None)
     ap.add_argument("--tile-bytes", type=int, default=None)
     ap.add_argument("--fused", type=int, default=None, help="plan key 'fused': 1, 0 or -1 (default)")
+    ap.add_argument("--custom", default=None, metavar="DTYPE,TOTAL_MIB,R,CHUNK_KIB",
+                    help="instead of a numbered config: one tensor per replica of that dtype (f32, bf16, ...), "
+                         "TOTAL_MIB over all R replicas, that chunk size, one flipped bit in the last replica "
+                         "(shape studies of the small-plan forms; not a headline workload)")
     ap.add_argument("--also", default=None,
                     help="comma-separated configs measured after the headline one and reported under "
                          "'also' (default: 3,5 for the default full-size run at N=1; '' for none)")
@@ -284,7 +288,15 @@ def run_config(cfg, args, rank, world, local, headline):
     import torch
     from paper_2608_11034_b200 import binding, dist_util, inputs
 
-    w = inputs.workload(cfg, BENCH_CASE.get(cfg, "default"), args.scale)
+    if args.custom and headline:
+        dtype, total_mib, R, chunk_kib = args.custom.split(",")
+        R = int(R)
+        numel = int(float(total_mib) * (1 << 20)) // R // inputs.DTYPE_BYTES[dtype]
+        w = inputs.Workload(f"custom_{dtype}_{total_mib}MiB_R{R}_chunk{chunk_kib}KiB", 0, "custom", R,
+                            int(chunk_kib) << 10, [inputs.TensorSpec("x", (numel,), dtype, "normal", 0.02)], 7)
+        w.patches = [inputs.Patch(R - 1, 0, numel // 2, "xor", 4)]
+    else:
+        w = inputs.workload(cfg, BENCH_CASE.get(cfg, "default"), args.scale)
     w.seed = dist_util.rank_seed(w.seed, rank)   # every rank scans its own replica set
     flats, views = inputs.generate(w, "cuda")
     total_bytes = w.R * w.bytes_per_replica
@@ -299,7 +311,7 @@ def run_config(cfg, args, rank, world, local, headline):
     if args.fused is not None:
         binding.scout_plan_set(plan.handle, "fused", args.fused)
     plan.bind(views)
-    use_certify = cfg == 4
+    use_certify = cfg == 4 and not args.custom
 
     def step():
         if use_certify:
@@ -392,6 +404,12 @@ def run_config(cfg, args, rank, world, local, headline):
             torch.cuda.synchronize()
             return sum(a0.elapsed_time(a1) for a0, a1 in evs) / args.steps
         one_launch = {"call": "scout_certify_launch (+ scout_certify_collect outside the timed pair)"}
+        # what an event pair costs on this machine with nothing, and with a trivial kernel, between
+        scratch = torch.zeros(32, device="cuda")
+        one_launch["event_pair_floor_ms"] = {"nothing": timed(lambda: None, lambda: None, False),
+                                             "torch_fill_of_128_bytes": timed(lambda: scratch.fill_(1.0),
+                                                                              lambda: None, False)}
+        one_launch["default_form"] = binding.scout_plan_get(plan.handle, "certify_form")
         for name, fused in (("one_kernel_clusters", 2), ("one_kernel", 1), ("kernel_per_stage", 0)):
             try:
                 binding.scout_plan_set(plan.handle, "fused", fused)
@@ -642,7 +660,7 @@ def main():
     # The other two large configs (bf16 parameters; 10,000 mixed tensors), measured the same
     # way after the headline config's buffers have been freed.
     if args.also is None:
-        also = [3, 5] if (args.config == 4 and args.scale == 1.0 and world == 1) else []
+        also = [3, 5] if (args.config == 4 and args.scale == 1.0 and world == 1 and not args.custom) else []
     else:
         also = [int(x) for x in args.also.split(",") if x]
     if also:

@@ -1453,7 +1453,8 @@ __global__ void __launch_bounds__(SIGN_THREADS, SCOUT_MINBLOCKS) certify_tiles(c
 // certificate chain, report) use global atomics, once per chunk.  The tile table is not
 // read: a chunk's tiles follow from its descriptor.  Chunks of fewer than 16 tiles are
 // taken `batch` at a time, so that every warp of a CTA has a tile.
-constexpr int CLUSTER_THREADS = 512;
+constexpr int CLUSTER_THREADS = 512;          // 256-thread CTAs measured equal or slower on every shape tried
+constexpr int CLUSTER_CTAS_PER_SM = 1024 / CLUSTER_THREADS;
 constexpr uint32_t CLUSTER_MAX_TILES = 512;   // records of one (chunk, replica) held in shared memory
 constexpr uint32_t CLUSTER_MAX_CTAS = 8;      // portable cluster size: R * split
 
@@ -1486,7 +1487,7 @@ __device__ __forceinline__ void st_cluster_record(uint32_t addr, const TileRec &
 }
 
 template <int DTSEL>
-__global__ void __launch_bounds__(CLUSTER_THREADS, 2) certify_clusters(const __grid_constant__ FusedArgs a) {
+__global__ void __launch_bounds__(CLUSTER_THREADS, CLUSTER_CTAS_PER_SM) certify_clusters(const __grid_constant__ FusedArgs a) {
     constexpr uint32_t WARPS = CLUSTER_THREADS / 32;
     __shared__ __align__(16) TileRec s_rec[CLUSTER_MAX_TILES];
     __shared__ uint64_t s_hash[WARPS][CLUSTER_MAX_CTAS];   // first CTA: hash of (chunk of the batch, replica)
@@ -1596,7 +1597,7 @@ int cluster_form_possible(int uniform_dtype, uint32_t R, uint32_t max_tiles, uin
     SCOUT_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
     const uint64_t clusters = (C + batch - 1) / batch;
     while (2 * split * R <= CLUSTER_MAX_CTAS && max_tiles >= 2 * split * WARPS &&
-           clusters * R * 2 * split <= 2ull * (uint64_t)sms)
+           clusters * R * 2 * split <= (uint64_t)CLUSTER_CTAS_PER_SM * (uint64_t)sms)
         split *= 2;
     *batch_out = batch;
     *split_out = split;
