@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libscout_b200.so")
-SOURCES = ["scout_api.cu", "scout_sign.cu", "scout_vote.cu", "scout_timing.cu", "scout_ledger.cpp"]
+SOURCES = ["scout_api.cu", "scout_sign.cu", "scout_one_launch.cu", "scout_noalloc.cu", "scout_vote.cu", "scout_timing.cu", "scout_ledger.cpp"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "-Xcompiler", "-fvisibility=hidden", "-Xlinker", "--exclude-libs,ALL"]
 
@@ -23,7 +23,7 @@ def _nvcc() -> str:
 
 def sources():
     srcs = [os.path.join(CSRC, s) for s in SOURCES]
-    deps = srcs + [os.path.join(CSRC, h) for h in ("scout_internal.h", "scout_vote_device.cuh")] + \
+    deps = srcs + [os.path.join(CSRC, h) for h in ("scout_internal.h", "scout_vote_device.cuh", "scout_scan.cuh", "scout_combine.cuh")] + \
         [os.path.join(ROOT, "include", h) for h in sorted(os.listdir(os.path.join(ROOT, "include")))]
     return srcs, deps
 

@@ -1,4 +1,4 @@
-// Compute-only cost of the scan's row routine (TileScan::row of scout_sign.cu): the rows
+// Compute-only cost of the scan's row routine (TileScan of scout_scan.cuh): the rows
 // come from shared memory (one 16-byte load per lane per row, as from global memory in the
 // real kernel), so no DRAM traffic is involved, and the kernel runs in the scan's launch
 // configuration: 256 threads per CTA, 1, 2 or 4 CTAs per SM (2, 4, 8 warps per scheduler).
@@ -12,9 +12,14 @@
 #include <cstdio>
 #include <cstdlib>
 
-#include "../scout_sign.cu"
-namespace scout { void set_cuda_error(cudaError_t, const char *) {} }
+#include "../scout_scan.cuh"
 using namespace scout;
+
+static __device__ __forceinline__ uint4 lds16(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
 
 template <int DT, int MODE>
 __global__ void __launch_bounds__(256, 4) rows(const uint4 *in, TileRec *out, int iters) {

@@ -1,6 +1,6 @@
 // Host side of the C ABI: plan construction (chunk and tile tables), argument
 // validation, launch sequencing, and the certify roll-up.  All arithmetic of the
-// method runs in the kernels of scout_sign.cu and scout_vote.cu.
+// method runs in the kernels of scout_sign.cu, scout_one_launch.cu, scout_noalloc.cu and scout_vote.cu.
 #include <algorithm>
 #include <cstdlib>
 #include <cstring>

@@ -189,7 +189,7 @@ struct SignLaunch {
 int launch_sign_tiles(const SignLaunch &a, cudaStream_t stream);
 
 // One launch for scan + finalise (mode 0), or scan + finalise + vote + certificate +
-// report (mode 1): see certify_tiles in scout_sign.cu.
+// report (mode 1): see certify_tiles and certify_clusters in scout_one_launch.cu.
 struct FusedLaunch {
     SignLaunch sign;            // the whole plan: tile_begin 0, every tile, every replica, ptrs set
     const ChunkDesc *chunks;    // device [C]
