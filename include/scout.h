@@ -292,9 +292,10 @@ SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/)
  *                     scan, finalise, vote, certificate - the form scout_certify_host
  *                     always uses).  -1 (default) = whichever measured fastest:
  *                     scout_certify on plans below 1 GiB uses clusters when R <= 8, no
- *                     chunk has more than 64 tiles and there are at most 1,024 chunks,
- *                     tickets on other plans up to 16 MiB; larger plans and
- *                     scout_sign_chunks run the stages as separate kernels
+ *                     chunk has more than 64 tiles per CTA that shares it and there are
+ *                     at most 1,024 chunks, tickets on other plans up to 16 MiB whose
+ *                     chunks have at most 64 tiles; larger plans and scout_sign_chunks
+ *                     run the stages as separate kernels
  *   get "certify_form", "sign_form"  the form (0, 1, 2 as above) scout_certify /
  *                     scout_sign_chunks would use for this plan now
  *   get "cluster_ok"  1 if form 2 can run this plan with its current tile size

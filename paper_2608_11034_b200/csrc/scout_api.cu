@@ -251,7 +251,8 @@ int upload_tables(scout_plan *p) {
 //     1 MiB chunks: 59-68 against 74-84 and 69-73.  With more chunks the sequential
 //     certificate chain (32 ns per chunk) decides and the per-stage form is as fast; with
 //     more tiles per chunk too few CTAs stream (an SM draws about 1/148 of the bandwidth).
-//   * scout_certify on other plans up to 16 MiB: tickets (29-35 us against 33-40).
+//   * scout_certify on other plans up to 16 MiB whose chunks have at most 64 tiles (in
+//     practice: more than 8 replicas): tickets (29-35 us against 33-40).
 //   * everything else: per stage.  With its work handed out dynamically the staged scan
 //     reaches 7.2 TB/s on 36 GB of fp32 and 6.5 TB/s on 125 GB of bf16; the ticket kernel
 //     stays 3 to 9 % below that, more than the three small launches it saves.
@@ -261,7 +262,7 @@ int launch_form(const scout_plan *p, bool certify) {
     if (p->fused == 1) return 1;
     if (!certify || p->total_bytes >= (1ull << 30)) return 0;
     if (p->cluster_ok && p->max_chunk_tiles <= 64 * p->cluster_split && p->chunks.size() <= 1024) return 2;
-    return p->total_bytes <= (16ull << 20) ? 1 : 0;
+    return (p->total_bytes <= (16ull << 20) && p->max_chunk_tiles <= 64) ? 1 : 0;
 }
 
 void fill_sign_launch(const scout_plan *p, SignLaunch &l) {

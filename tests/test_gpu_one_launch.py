@@ -200,7 +200,7 @@ def test_cluster_form_with_one_to_eight_replicas_and_the_limits():
 
 def test_the_default_picks_the_form_by_shape():
     """Key "fused" = -1: clusters for small plans of few-tile chunks and R <= 8, tickets for other
-    plans up to 16 MiB, one kernel per stage otherwise; scout_sign_chunks always per stage."""
+    plans of few-tile chunks up to 16 MiB, one kernel per stage otherwise; scout_sign_chunks always per stage."""
     from paper_2608_11034_b200 import binding as B
     def form(R, numel, chunk_bytes, dtype="f32"):
         w = inputs.Workload("p", 0, "x", R, chunk_bytes, [inputs.TensorSpec("x", (numel,), dtype, "normal", 1.0)], 3)
@@ -210,7 +210,7 @@ def test_the_default_picks_the_form_by_shape():
         return f
     assert form(3, 1 << 20, 65536) == (2, 0)            # 12.6 MB, 16 tiles per chunk
     assert form(4, 25_165_824, 1 << 20, "bf16") == (2, 0)   # 201 MB in 1 MiB chunks, 64 tiles per chunk
-    assert form(16, 1 << 18, 65536) == (1, 0)           # 16 replicas: no cluster; 16.8 MB... tickets up to 16 MiB
-    assert form(3, 1 << 20, 4 << 20) == (1, 0)          # one chunk of 1,024 tiles, 12.6 MB: tickets
+    assert form(16, 1 << 18, 65536) == (1, 0)           # 16 replicas of 1 MiB (16 MiB in all): no cluster, tickets
+    assert form(3, 1 << 20, 4 << 20) == (0, 0)          # one chunk of 1,024 tiles, 12.6 MB: per stage
     assert form(3, 16 << 20, 4 << 20) == (0, 0)         # 201 MB in 4 MiB chunks (256 tiles each): per stage
     assert form(3, 2 << 20, 2048) == (0, 0)             # 4,096 chunks: the chain decides, per stage
