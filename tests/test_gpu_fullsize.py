@@ -145,6 +145,43 @@ def test_configs_1_and_2_every_chunk(cfg, case):
     _free()
 
 
+@pytest.mark.parametrize("cfg,case", [(1, "default"), (2, "mantissa"), (2, "split22"), (2, "split211")])
+def test_configs_1_and_2_certify_in_the_default_form(cfg, case):
+    """scout_certify as the library launches it by default on these plans (one kernel, a
+    thread-block cluster per chunk): report, lists and every record against the oracle."""
+    from paper_2608_11034_b200 import binding
+    w = inputs.workload(cfg, case)
+    _, views = inputs.generate(w, "cuda")
+    host = [[v.cpu() for v in rep] for rep in views]
+    osigs, chunks = helpers.oracle_sign_all(w, host, nthreads=8)
+    want = orc.certify(osigs)
+    plan = helpers.gpu_plan(w)
+    assert binding.scout_plan_get(plan.handle, "certify_form") == 2
+    assert binding.scout_plan_get(plan.handle, "certify_kernels") == 1
+    plan.bind(views)
+    for _ in range(2):
+        got = plan.certify()
+        assert got["report"] == want["report"]
+        assert got["outliers"] == want["outliers"] and got["undecided"] == want["undecided"]
+    # the records that run left in the plan: their hashes enter the tensor roll-ups
+    d_sigs, _, _ = binding.scout_plan_results(plan.handle)
+    d_roll = torch.empty(len(w.specs) * w.R, dtype=torch.int64, device="cuda")
+    binding.scout_rollup_tensors(plan.handle, d_sigs, d_roll.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    roll = d_roll.cpu().numpy().view(np.uint64).reshape(len(w.specs), w.R)
+    for r in range(w.R):
+        assert int(roll[0, r]) == orc.rollup(osigs["hash"][:, r])
+    # and the same kernel as scout_sign_chunks: full records, sums included
+    binding.scout_plan_set(plan.handle, "fused", 2)
+    plan.sign()
+    torch.cuda.synchronize()
+    got_sigs = plan.d_sigs.cpu().numpy().view(binding.SIG_DTYPE).reshape(plan.C, w.R)
+    helpers.assert_sigs_match(got_sigs, osigs, helpers.chunk_abs_sums(w, host, chunks))
+    helpers.assert_guards(plan)
+    plan.close()
+    del views
+    _free()
+
+
 def test_config_4_certify_full_size():
     from paper_2608_11034_b200 import binding
     _free()
