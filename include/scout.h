@@ -291,9 +291,10 @@ SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/)
  *                     are taken several at a time.  0 = never (one kernel per stage:
  *                     scan, finalise, vote, certificate - the form scout_certify_host
  *                     always uses).  -1 (default) = whichever measured fastest:
- *                     scout_certify on plans below 1 GiB uses clusters when R <= 8, no
- *                     chunk has more than 64 tiles per CTA that shares it and there are
- *                     at most 1,024 chunks, tickets on other plans up to 16 MiB whose
+ *                     scout_certify on plans below 1 GiB (256 MiB for plans of 16-bit
+ *                     floats) uses clusters when R <= 8, no chunk has more than 64 tiles
+ *                     per CTA that shares it and there are at most 1,024 chunks (or one
+ *                     per 300 KiB), tickets on other plans up to 16 MiB whose
  *                     chunks have at most 64 tiles; larger plans and scout_sign_chunks
  *                     run the stages as separate kernels
  *   get "certify_form", "sign_form"  the form (0, 1, 2 as above) scout_certify /

@@ -248,9 +248,12 @@ int upload_tables(scout_plan *p) {
 //   * scout_certify on a plan below 1 GiB whose chunks have at most 64 tiles and which has
 //     at most 1,024 chunks, R <= 8: clusters.  12.6 MB in 64 KiB chunks: 25 us against 29
 //     (tickets) and 33 (per stage); 50 MB in 256 KiB chunks: 33 against 57 and 46; 201 MB in
-//     1 MiB chunks: 59-68 against 74-84 and 69-73.  With more chunks the sequential
-//     certificate chain (32 ns per chunk) decides and the per-stage form is as fast; with
-//     more tiles per chunk too few CTAs stream (an SM draws about 1/148 of the bandwidth).
+//     1 MiB chunks: 59-68 against 74-84 and 69-73; 900 MiB in 1 MiB chunks: 188 against 204
+//     and 191.  With more chunks (1,024, or one per 300 KiB of the plan if that is more) the
+//     sequential certificate chain (32 ns per chunk) decides and the per-stage form is as
+//     fast; with more tiles per chunk too few CTAs stream (a CTA has 64 KiB in flight, about
+//     50 GB/s).  Plans of 16-bit floats above 256 MiB: per stage (their row routine bounds an
+//     SM at 47-49 GB/s, so the uneven spread of CTAs over SMs costs 11 % at 900 MiB).
 //   * scout_certify on other plans up to 16 MiB whose chunks have at most 64 tiles (in
 //     practice: more than 8 replicas): tickets (29-35 us against 33-40).
 //   * everything else: per stage.  With its work handed out dynamically the staged scan
@@ -261,7 +264,11 @@ int launch_form(const scout_plan *p, bool certify) {
     if (p->fused == 2) return p->cluster_ok ? 2 : 1;
     if (p->fused == 1) return 1;
     if (!certify || p->total_bytes >= (1ull << 30)) return 0;
-    if (p->cluster_ok && p->max_chunk_tiles <= 64 * p->cluster_split && p->chunks.size() <= 1024) return 2;
+    const bool half_floats = p->uniform_dtype == SCOUT_DT_BF16 || p->uniform_dtype == SCOUT_DT_F16;
+    const uint64_t max_chunks = std::max<uint64_t>(1024, p->total_bytes / (300ull << 10));
+    if (p->cluster_ok && p->max_chunk_tiles <= 64 * p->cluster_split && p->chunks.size() <= max_chunks &&
+        (!half_floats || p->total_bytes <= (256ull << 20)))
+        return 2;
     return (p->total_bytes <= (16ull << 20) && p->max_chunk_tiles <= 64) ? 1 : 0;
 }
 
