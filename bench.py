@@ -88,6 +88,7 @@ def parse_args():
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--variant", type=int, default=None)
     ap.add_argument("--tile-bytes", type=int, default=None)
+    ap.add_argument("--work-streams", type=int, default=None, help="plan key 'work_streams'")
     ap.add_argument("--fused", type=int, default=None, help="plan key 'fused': 1, 0 or -1 (default)")
     ap.add_argument("--custom", default=None, metavar="DTYPE,TOTAL_MIB,R,CHUNK_KIB",
                     help="instead of a numbered config: one tensor per replica of that dtype (f32, bf16, ...), "
@@ -310,6 +311,8 @@ def run_config(cfg, args, rank, world, local, headline):
         binding.scout_plan_set(plan.handle, "variant", args.variant)
     if args.fused is not None:
         binding.scout_plan_set(plan.handle, "fused", args.fused)
+    if args.work_streams is not None:
+        binding.scout_plan_set(plan.handle, "work_streams", args.work_streams)
     plan.bind(views)
     use_certify = cfg == 4 and not args.custom
 

@@ -300,8 +300,11 @@ SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/)
  *   get "certify_form", "sign_form"  the form (0, 1, 2 as above) scout_certify /
  *                     scout_sign_chunks would use for this plan now
  *   get "cluster_ok"  1 if form 2 can run this plan with its current tile size
- *   set "dynamic"     1 (default): the scan's warps take tiles from a work counter as they
+ *   set "dynamic"     1 (default): the scan's warps take tiles from work counters as they
  *                     become free; 0: fixed round-robin assignment
+ *   set "work_streams" 1..32 (default 8): how many counters the tiles are dealt from (one
+ *                     counter serves about 0.3 G tiles per second, which plans of many
+ *                     small tiles exceed)
  *   set "grid"        CTAs of the scan kernel
  *   set "timing"      1: record a pair of CUDA events around every scan kernel on
  *                     the caller's stream (a ring of 256 pairs); setting it again

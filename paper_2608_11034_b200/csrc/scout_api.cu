@@ -35,6 +35,8 @@ static uint32_t dtype_size(uint32_t d) {
 
 using namespace scout;
 
+constexpr uint32_t MAX_WORK_STREAMS = 32;  // work counters of the direct scan: [2][streams], 128 bytes apart
+constexpr size_t WORK_BYTES = 2 * MAX_WORK_STREAMS * 128;
 constexpr size_t TIMING_RING = 256;  // event pairs kept for the "timing" knob
 
 struct scout_plan {
@@ -81,6 +83,9 @@ struct scout_plan {
     unsigned long long *d_work2 = nullptr;  // direct scan kernels of the staged path
     uint64_t work_launches = 0;
     bool dynamic = true;                    // key "dynamic"
+    uint32_t work_streams = 8;              // key "work_streams": counters the tiles are dealt from (one
+                                            // counter hands out about 0.3 G tiles/s: 3 GB in 4 KiB chunks
+                                            // scans at 1.8 TB/s with one counter, 5.9 TB/s with eight)
     CertifyHost *h_out_dev = nullptr;  // device-side address of h_out
     uint32_t epoch = 0;
     bool out_dirty = false;       // d_out was left non-zero by the multi-kernel path
@@ -290,6 +295,7 @@ void fill_sign_launch(const scout_plan *p, SignLaunch &l) {
     l.grid = p->grid;
     l.work = nullptr;
     l.work_parity = 0;
+    l.work_streams = 1;
 }
 
 // The direct scan kernels take their work dynamically: successive launches alternate between
@@ -297,6 +303,7 @@ void fill_sign_launch(const scout_plan *p, SignLaunch &l) {
 void next_work_counter(scout_plan *p, SignLaunch &l) {
     l.work = p->dynamic ? p->d_work2 : nullptr;
     l.work_parity = (p->work_launches++) & 1u;
+    l.work_streams = p->work_streams;
 }
 
 // One kernel: scan + finalise (certify == false), or the whole certify path.  The timing
@@ -575,7 +582,7 @@ int scout_plan_create(uint32_t R, uint64_t T, const scout_tensor_t *tensors, uin
             plan_malloc(p, (void **)&p->d_done, nc * sizeof(uint32_t)) != cudaSuccess ||
             plan_malloc(p, (void **)&p->d_chain, sizeof(ChainState)) != cudaSuccess ||
             plan_malloc(p, (void **)&p->d_work, 2 * sizeof(unsigned long long)) != cudaSuccess ||
-            plan_malloc(p, (void **)&p->d_work2, 2 * sizeof(unsigned long long)) != cudaSuccess) {
+            plan_malloc(p, (void **)&p->d_work2, WORK_BYTES) != cudaSuccess) {
             rc = SCOUT_ERR_NOMEM;
             break;
         }
@@ -583,7 +590,7 @@ int scout_plan_create(uint32_t R, uint64_t T, const scout_tensor_t *tensors, uin
             cudaMemset(p->d_done, 0, nc * sizeof(uint32_t)) != cudaSuccess ||
             cudaMemset(p->d_chain, 0, sizeof(ChainState)) != cudaSuccess ||
             cudaMemset(p->d_work, 0, 2 * sizeof(unsigned long long)) != cudaSuccess ||
-            cudaMemset(p->d_work2, 0, 2 * sizeof(unsigned long long)) != cudaSuccess) {
+            cudaMemset(p->d_work2, 0, WORK_BYTES) != cudaSuccess) {
             rc = SCOUT_ERR_CUDA;
             break;
         }
@@ -900,6 +907,13 @@ int scout_plan_set(scout_plan_t *p, const char *key, int64_t value) {
         }
         return upload_tables(p);
     }
+    if (!std::strcmp(key, "work_streams")) {
+        if (value < 1 || value > (int64_t)MAX_WORK_STREAMS) return SCOUT_ERR_INVALID;
+        if (p->launched) SCOUT_CUDA(cudaEventSynchronize(p->ev_last));   // the counters may be in use
+        p->work_streams = (uint32_t)value;
+        SCOUT_CUDA(cudaMemset(p->d_work2, 0, WORK_BYTES));
+        return SCOUT_OK;
+    }
     if (!std::strcmp(key, "dynamic")) {
         p->dynamic = value != 0;
         return SCOUT_OK;
@@ -954,6 +968,7 @@ int scout_plan_get(const scout_plan_t *p, const char *key, int64_t *value) {
         return guards_intact(p, value);
     }
     else if (!std::strcmp(key, "fused")) *value = p->fused;
+    else if (!std::strcmp(key, "work_streams")) *value = p->work_streams;
     else if (!std::strcmp(key, "certify_form")) *value = launch_form(p, true);
     else if (!std::strcmp(key, "sign_form")) *value = launch_form(p, false);
     else if (!std::strcmp(key, "cluster_ok")) *value = p->cluster_ok;

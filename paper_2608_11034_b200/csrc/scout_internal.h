@@ -182,8 +182,10 @@ struct SignLaunch {
     uint32_t *error;              // device flag set when a bounded wait gave up (may be null)
     int variant;                  // 0 direct, 1 direct + register prefetch, 2 bulk-async ring, 3 read probe
     int uniform_dtype;            // dtype shared by every tile of the launch, or -1 if they differ
-    unsigned long long *work;     // device [2] work counters of the direct scan (null: fixed round-robin)
+    unsigned long long *work;     // device [2][work_streams] work counters of the direct scan, 128 bytes
+                                  // apart (null: fixed round-robin)
     uint32_t work_parity;         // which of the two this launch uses (successive launches alternate)
+    uint32_t work_streams;        // counters the items are dealt from (0 or 1: one), 128 bytes apart
     int grid;                     // CTAs to launch
 };
 int launch_sign_tiles(const SignLaunch &a, cudaStream_t stream);

@@ -480,6 +480,7 @@ int launch_fused(const FusedLaunch &l, cudaStream_t stream) {
     a.s.error = l.sign.error;
     a.s.work = nullptr;
     a.s.work_parity = 0;
+    a.s.work_streams = 1;
     a.chunks = l.chunks;
     a.C = l.C;
     a.R = l.R;

@@ -404,6 +404,7 @@ struct SignArgs {
     // successive launches (null: static round-robin), and this launch's parity
     unsigned long long *work;
     uint32_t work_parity;
+    uint32_t work_streams; // counters the items are dealt from (>= 1)
 };
 
 __device__ __forceinline__ void scan_dispatch(uint32_t dtype, const uint8_t *tile, uint32_t nbytes,

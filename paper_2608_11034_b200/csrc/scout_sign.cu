@@ -9,6 +9,58 @@
 namespace scout {
 namespace {
 
+// Work distribution of the direct scan and of the read probe.  Every warp starts with item
+// `warp`; the items after the first n_warps are handed out as warps become free (tiles differ
+// in size and dtype, and SMs differ in how the memory system serves them, so a fixed
+// round-robin ends with its slowest warp).  They are dealt from `streams` counters, 128 bytes
+// apart: counter j hands out the items n_warps + j, n_warps + j + streams, ... in order, and a
+// warp draws from counter (warp mod streams) until that one has run out, then from the next.
+// One counter is one address, served by one L2 slice at about one atomic per 3 ns, which is
+// about the rate at which a B200 finishes 32 KiB tiles; several counters keep the hand-out
+// off that limit while the tiles in flight stay one contiguous window of the input (claiming
+// several consecutive tiles per atomic was tried instead and cost 2-5 %).  The request for the
+// next item is made before the current tile is scanned and its answer is read after it.  The
+// counters of this launch are those of work_parity; the others are zeroed here for the launch
+// that follows.
+constexpr uint32_t WORK_STRIDE = 16;   // 64-bit words between two counters (128 bytes)
+struct WorkQueue {
+    unsigned long long *ctr;   // this launch's counters, or null: fixed round-robin
+    uint64_t n_warps, n_items, n_rest;
+    uint32_t streams, stream, empty_seen;
+
+    __device__ __forceinline__ void begin(const SignArgs &a, uint64_t warp, uint64_t warps, uint64_t items,
+                                          uint32_t lane) {
+        n_warps = warps;
+        n_items = items;
+        n_rest = items > warps ? items - warps : 0;
+        streams = a.work_streams;
+        ctr = (a.work && n_rest) ? a.work + (uint64_t)a.work_parity * streams * WORK_STRIDE : nullptr;
+        if (a.work && warp == 0 && lane < streams)
+            a.work[((uint64_t)(a.work_parity ^ 1u) * streams + lane) * WORK_STRIDE] = 0ull;
+        stream = (uint32_t)(warp % streams);
+        empty_seen = 0;
+    }
+    // lane 0: ask for the next item (the answer is used by next_item)
+    __device__ __forceinline__ unsigned long long request(uint32_t lane) const {
+        unsigned long long k = 0;
+        if (ctr && lane == 0) k = atomicAdd(ctr + stream * WORK_STRIDE, 1ull);
+        return k;
+    }
+    // the item that follows `item`, given the answer to the request made before it was scanned
+    __device__ __forceinline__ uint64_t next_item(uint64_t item, unsigned long long answer, uint32_t lane) {
+        if (!ctr) return item + n_warps;
+        uint64_t i = __shfl_sync(0xFFFFFFFFu, answer, 0) * streams + stream;
+        while (i >= n_rest) {   // this counter has run out: the next one (only at the very end of a launch)
+            if (++empty_seen >= streams) return n_items;
+            stream = stream + 1 == streams ? 0 : stream + 1;
+            unsigned long long k = 0;
+            if (lane == 0) k = atomicAdd(ctr + stream * WORK_STRIDE, 1ull);
+            i = __shfl_sync(0xFFFFFFFFu, k, 0) * streams + stream;
+        }
+        return n_warps + i;
+    }
+};
+
 // Persistent grid; every warp takes whole tiles, replica-major, round-robin.
 // DTSEL >= 0: every tile of the launch has that dtype (the element path is fixed at
 // compile time, so the register allocation is that path's, not the union of all
@@ -18,22 +70,11 @@ __global__ void __launch_bounds__(SIGN_THREADS, PREFETCH ? SCOUT_MINBLOCKS_PF : 
     pdl_launch_dependents();
     const uint32_t lane = threadIdx.x & 31u;
     const uint64_t warp = (uint64_t)blockIdx.x * (SIGN_THREADS / 32) + (threadIdx.x >> 5);
-    const uint64_t n_warps = (uint64_t)gridDim.x * (SIGN_THREADS / 32);
-    const uint64_t n_items = a.n_tiles * a.n_replicas;
-    // Every warp starts with item `warp`.  With a work counter the later items are handed out
-    // in order as warps become free (tiles differ in size and dtype, so a fixed round-robin
-    // leaves some warps with more bytes than others); the request for the next item is made
-    // before the current tile is scanned and its answer is read after it.  The counter of this
-    // launch is work[parity]; the other one is zeroed here for the launch that follows.
-    unsigned long long *work = a.work ? a.work + a.work_parity : nullptr;
-    if (work && warp == 0 && lane == 0) a.work[a.work_parity ^ 1u] = 0ull;
-    const bool dynamic = work != nullptr && n_items > n_warps;
+    WorkQueue q;
+    q.begin(a, warp, (uint64_t)gridDim.x * (SIGN_THREADS / 32), a.n_tiles * a.n_replicas, lane);
     uint64_t item = warp;
-    while (item < n_items) {
-        unsigned long long next = 0;
-        if (dynamic) {
-            if (lane == 0) next = atomicAdd(work, 1ull);
-        }
+    while (item < q.n_items) {
+        const unsigned long long answer = q.request(lane);
         const uint32_t rr = (uint32_t)(item / a.n_tiles);
         const uint64_t t = a.tile_begin + (item - (uint64_t)rr * a.n_tiles);
         const uint32_t r = a.replica_begin + rr;
@@ -48,7 +89,7 @@ __global__ void __launch_bounds__(SIGN_THREADS, PREFETCH ? SCOUT_MINBLOCKS_PF : 
             else          scan_dispatch(td.dtype, tile, td.nbytes, lane, rec);
         }
         if (lane == 0) store_record(&a.recs[(uint64_t)r * a.tiles_per_replica + t], rec);
-        item = dynamic ? n_warps + __shfl_sync(0xFFFFFFFFu, next, 0) : item + n_warps;
+        item = q.next_item(item, answer, lane);
     }
 }
 
@@ -549,18 +590,11 @@ __global__ void bounded_wait_selftest(unsigned long long limit_ns, unsigned long
 __global__ void __launch_bounds__(SIGN_THREADS) read_probe(const SignArgs a) {
     const uint32_t lane = threadIdx.x & 31u;
     const uint64_t warp = (uint64_t)blockIdx.x * (SIGN_THREADS / 32) + (threadIdx.x >> 5);
-    const uint64_t n_warps = (uint64_t)gridDim.x * (SIGN_THREADS / 32);
-    const uint64_t n_items = a.n_tiles * a.n_replicas;
-    // the same work distribution as the scan (see sign_tiles_direct)
-    unsigned long long *work = a.work ? a.work + a.work_parity : nullptr;
-    if (work && warp == 0 && lane == 0) a.work[a.work_parity ^ 1u] = 0ull;
-    const bool dynamic = work != nullptr && n_items > n_warps;
+    WorkQueue q;   // the same work distribution as the scan
+    q.begin(a, warp, (uint64_t)gridDim.x * (SIGN_THREADS / 32), a.n_tiles * a.n_replicas, lane);
     uint64_t item = warp;
-    while (item < n_items) {
-        unsigned long long next = 0;
-        if (dynamic) {
-            if (lane == 0) next = atomicAdd(work, 1ull);
-        }
+    while (item < q.n_items) {
+        const unsigned long long answer = q.request(lane);
         const uint32_t rr = (uint32_t)(item / a.n_tiles);
         const uint64_t t = a.tile_begin + (item - (uint64_t)rr * a.n_tiles);
         const uint32_t r = a.replica_begin + rr;
@@ -584,7 +618,7 @@ __global__ void __launch_bounds__(SIGN_THREADS) read_probe(const SignArgs a) {
 #pragma unroll
         for (int d = 16; d >= 1; d >>= 1) y ^= __shfl_xor_sync(0xFFFFFFFFu, y, d);
         if (lane == 0) a.recs[(uint64_t)r * a.tiles_per_replica + t].h = y;
-        item = dynamic ? n_warps + __shfl_sync(0xFFFFFFFFu, next, 0) : item + n_warps;
+        item = q.next_item(item, answer, lane);
     }
 }
 
@@ -651,6 +685,7 @@ int launch_sign_tiles(const SignLaunch &l, cudaStream_t stream) {
     a.error = l.error;
     a.work = l.work;
     a.work_parity = l.work_parity;
+    a.work_streams = l.work_streams ? l.work_streams : 1u;
     const uint64_t items = l.n_tiles * l.n_replicas;
     const uint64_t want = (items + SIGN_THREADS / 32 - 1) / (SIGN_THREADS / 32);
     int grid = l.grid;

@@ -231,3 +231,31 @@ def test_guard_bands_notice_a_stray_write():
     outer[B.Plan.GUARD_BYTES - 1] = B.Plan.GUARD_PATTERN
     assert plan.check_guards()
     plan.close()
+
+
+@pytest.mark.parametrize("streams", [1, 3, 8, 32])
+def test_work_counters_any_number_same_records(streams):
+    """The tiles of the staged scan are dealt from `work_streams` counters; a warp whose counter
+    has run out moves on to the next.  Whatever their number, every tile is scanned exactly once:
+    records equal to the oracle's, twice in a row (the counters of one launch are zeroed by the
+    previous one).  13,000 tiles for 4,736 warps, so most tiles come from the counters."""
+    from paper_2608_11034_b200 import binding as b
+    spec = inputs.TensorSpec("x", (2_218_667,), "f32", "normal", 0.02)      # 4,334 tiles of 2 KiB per replica
+    w = inputs.Workload("streams", 0, "x", 3, 65536, [spec], 31)
+    w.patches = [inputs.Patch(2, 0, 2_000_000, "xor", 1 << 7)]
+    _, views = inputs.generate(w, "cuda")
+    host = [[v.cpu() for v in rep] for rep in views]
+    osigs, chunks = helpers.oracle_sign_all(w, host)
+    plan = helpers.gpu_plan(w, tile_bytes=2048, variant="unfused")
+    b.scout_plan_set(plan.handle, "work_streams", streams)
+    assert b.scout_plan_get(plan.handle, "work_streams") == streams
+    plan.bind(views)
+    for _ in range(3):
+        plan.sign()
+        torch.cuda.synchronize()
+        gs = plan.d_sigs.cpu().numpy().view(b.SIG_DTYPE).reshape(plan.C, w.R)
+        helpers.assert_sigs_match(gs, osigs, helpers.chunk_abs_sums(w, host, chunks))
+    with pytest.raises(b.ScoutError):
+        b.scout_plan_set(plan.handle, "work_streams", 33)
+    helpers.assert_guards(plan)
+    plan.close()
