@@ -634,15 +634,30 @@ __global__ void __launch_bounds__(FIN_THREADS) finalize_chunks(const ChunkDesc *
     const uint32_t lane = threadIdx.x & 31u;
     const uint64_t warp = (uint64_t)blockIdx.x * (FIN_THREADS / 32) + (threadIdx.x >> 5);
     const uint64_t n_warps = (uint64_t)gridDim.x * (FIN_THREADS / 32);
-    for (uint64_t item = warp; item < C * R; item += n_warps) {
-        const uint64_t c = item / R;
-        const uint32_t r = (uint32_t)(item - c * R);
+    // One item = one chunk and up to COMBINE_BATCH replicas of it: the chunk's geometry (its
+    // descriptor, the lanes' weights) is worked out once for them, and for chunks of at most
+    // 32 tiles their record loads are in flight together (a warp's items are a chain of
+    // dependent memory round trips, so fewer and wider items are what shortens the kernel).
+    const uint32_t groups = (R + COMBINE_BATCH - 1) / COMBINE_BATCH;
+    for (uint64_t item = warp; item < C * groups; item += n_warps) {
+        const uint64_t c = item / groups;
+        const uint32_t r0 = (uint32_t)(item - c * groups) * COMBINE_BATCH;
+        const uint32_t n_rep = min((uint32_t)COMBINE_BATCH, R - r0);
         const ChunkDesc cd = chunks[c];
-        const scout_sig_t o = combine_tiles(recs + (uint64_t)r * tiles_per_replica + cd.tile0, cd.ntiles,
-                                            cd.nbytes, cd.k, cd.dtype, cd.meta, p_stride,
-                                            combine_weight(cd.ntiles, cd.nbytes, tile_rows, lane), lane);
-        if (lane == 0) {
-            sigs[c * R + r] = o;
+        const uint64_t weight = combine_weight(cd.ntiles, cd.nbytes, tile_rows, lane);
+        const TileRec *tr = recs + (uint64_t)r0 * tiles_per_replica + cd.tile0;
+        if (cd.ntiles <= 32u) {
+            scout_sig_t o[COMBINE_BATCH];
+            combine_small(tr, tiles_per_replica, n_rep, cd.ntiles, cd.nbytes, cd.k, cd.dtype, cd.meta, weight, lane, o);
+#pragma unroll
+            for (int j = 0; j < COMBINE_BATCH; ++j)
+                if ((uint32_t)j < n_rep && lane == 0) sigs[c * R + r0 + j] = o[j];
+        } else {
+            for (uint32_t j = 0; j < n_rep; ++j) {
+                const scout_sig_t o = combine_tiles(tr + (uint64_t)j * tiles_per_replica, cd.ntiles, cd.nbytes, cd.k,
+                                                    cd.dtype, cd.meta, p_stride, weight, lane);
+                if (lane == 0) sigs[c * R + r0 + j] = o;
+            }
         }
     }
 }
@@ -716,7 +731,7 @@ int launch_finalize(const ChunkDesc *chunks, uint64_t C, uint32_t R, const TileR
                     uint64_t tiles_per_replica, uint32_t tile_rows, scout_sig_t *d_sigs,
                     CertifyOut *zero_out, cudaStream_t stream) {
     if (C == 0) return SCOUT_OK;
-    const uint64_t items = C * R;
+    const uint64_t items = C * ((R + COMBINE_BATCH - 1) / COMBINE_BATCH);
     uint64_t blocks = (items + FIN_THREADS / 32 - 1) / (FIN_THREADS / 32);
     if (blocks > 148ull * 16) blocks = 148ull * 16;
     static_assert(sizeof(CertifyOut) / sizeof(uint64_t) <= FIN_THREADS, "one thread per word clears it");
