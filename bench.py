@@ -50,7 +50,7 @@ SCAN_TRAFFIC_SOURCE = ("ncu capture of the scan kernel on 1.8 GB at commit 50ceb
 # SM cycles per 512-byte row and scheduler of the scan's row routine with its data already on the
 # SM (`python -m paper_2608_11034_b200.microbench`, its output is summarised under profiles/): the
 # compute bound of a uniform-dtype workload at SM clock f is 512 B * 4 * SMs * f / cycles.
-ROW_COST_CYCLES = {"bf16": 81.4, "f16": 81.3, "f32": 51.4, "i64": 41.3, "u8": 26.9}
+ROW_COST_CYCLES = {"bf16": 74.8, "f16": 74.7, "f32": 44.6, "i64": 41.4, "u8": 26.9}
 N_SMS = 148
 
 
@@ -294,7 +294,10 @@ def run_config(cfg, args, rank, world, local, headline):
         R = int(R)
         numel = int(float(total_mib) * (1 << 20)) // R // inputs.DTYPE_BYTES[dtype]
         w = inputs.Workload(f"custom_{dtype}_{total_mib}MiB_R{R}_chunk{chunk_kib}KiB", 0, "custom", R,
-                            int(chunk_kib) << 10, [inputs.TensorSpec("x", (numel,), dtype, "normal", 0.02)], 7)
+                            int(chunk_kib) << 10,
+                            [inputs.TensorSpec("x", (numel,), dtype,
+                                               {"u8": "bytes", "i64": "randint40", "i32": "randfull"}.get(dtype, "normal"),
+                                               0.02)], 7)
         w.patches = [inputs.Patch(R - 1, 0, numel // 2, "xor", 4)]
     else:
         w = inputs.workload(cfg, BENCH_CASE.get(cfg, "default"), args.scale)

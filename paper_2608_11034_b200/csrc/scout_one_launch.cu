@@ -263,7 +263,7 @@ __global__ void __launch_bounds__(SIGN_THREADS, SCOUT_MINBLOCKS) certify_tiles(c
         // whoever completes this chunk reads its descriptor: have it in L2 by then
         if (lane == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(a.chunks + td.chunk));
         TileRec rec;
-        if constexpr (DTSEL >= 0) scan_tile<DTSEL>(tile, td.nbytes, lane, rec);
+        if constexpr (DTSEL >= 0) scan_tile<DTSEL, true>(tile, td.nbytes, lane, rec);
         else                      scan_dispatch(td.dtype, tile, td.nbytes, lane, rec);
         if (prev_tiles) resolve_ticket(a, lane, prev_returned, prev_tiles, prev_chunk);
         if (lane == 0) {
@@ -360,7 +360,7 @@ __global__ void __launch_bounds__(CLUSTER_THREADS, CLUSTER_CTAS_PER_SM) certify_
             const uint64_t off = (uint64_t)j * tile_bytes;
             const uint32_t nbytes = (uint32_t)min((uint64_t)tile_bytes, cd.nbytes - off);
             TileRec rec;
-            if constexpr (DTSEL >= 0) scan_tile<DTSEL>(base + off, nbytes, lane, rec);
+            if constexpr (DTSEL >= 0) scan_tile<DTSEL, true>(base + off, nbytes, lane, rec);
             else                      scan_dispatch(cd.dtype, base + off, nbytes, lane, rec);
             if (lane == 0) {
                 if (split > 1) st_cluster_record(home + (slot0 + j) * (uint32_t)sizeof(TileRec), rec);

@@ -253,22 +253,46 @@ __device__ __noinline__ void rescan_classifying(const uint8_t *tile, uint32_t nb
 }
 
 // h <- h * P + (m0 w0 + m1 w1 + m2 w2 + m3 w3) mod 2^64.  Starting the chain from
-// h * P lets every product be a 32x32+64 multiply-add (measured: fewest
-// instructions of the forms tried; a 64-bit accumulate costs two issue slots).
+// h * P lets every product be a 32x32+64 multiply-add.  Two spellings of the same
+// arithmetic.  From the C++ expression the compiler makes 11 instructions per row; from
+// the PTX chain the 7 it needs (one wide multiply and two 32-bit multiply-adds for h * P,
+// four wide multiply-adds).  Which one is faster depends on what surrounds it (measured
+// in one session, 3 GB to 125 GB per step): in the kernels compiled for a single element
+// type the PTX chain wins (fp32 6,905-6,918 -> 7,027-7,034 GB/s, bf16 6,352-6,381 ->
+// 6,470-6,490), in the kernel that reads the type from the tile table the C++ form does
+// (int64 7,198 against 7,009, uint8 7,194 / 6,990, int32 7,175 / 6,799, fp64 6,883 /
+// 6,803; mixed fp32/bf16/int64 equal).  So PTX_CHAIN is set by the single-type kernels only.
+template <bool PTX_CHAIN>
 __device__ __forceinline__ void fold_row(uint64_t &h, const uint4 &v, const uint32_t (&m)[4]) {
-    uint64_t t = h * HASH_P;
-    t += (uint64_t)m[0] * v.x;
-    t += (uint64_t)m[1] * v.y;
-    t += (uint64_t)m[2] * v.z;
-    t += (uint64_t)m[3] * v.w;
-    h = t;
+    if constexpr (PTX_CHAIN) {
+        const uint32_t lo = (uint32_t)h, hi = (uint32_t)(h >> 32);
+        constexpr uint32_t P_LO = (uint32_t)HASH_P, P_HI = (uint32_t)(HASH_P >> 32);
+        uint64_t t;
+        uint32_t th;
+        asm("mul.wide.u32 %0, %1, %2;" : "=l"(t) : "r"(lo), "r"(P_LO));
+        asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(th) : "r"(lo), "r"(P_HI), "r"((uint32_t)(t >> 32)));
+        asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(th) : "r"(hi), "r"(P_LO), "r"(th));
+        t = ((uint64_t)th << 32) | (uint32_t)t;
+        asm("mad.wide.u32 %0, %1, %2, %0;" : "+l"(t) : "r"(m[0]), "r"(v.x));
+        asm("mad.wide.u32 %0, %1, %2, %0;" : "+l"(t) : "r"(m[1]), "r"(v.y));
+        asm("mad.wide.u32 %0, %1, %2, %0;" : "+l"(t) : "r"(m[2]), "r"(v.z));
+        asm("mad.wide.u32 %0, %1, %2, %0;" : "+l"(t) : "r"(m[3]), "r"(v.w));
+        h = t;
+    } else {
+        uint64_t t = h * HASH_P;
+        t += (uint64_t)m[0] * v.x;
+        t += (uint64_t)m[1] * v.y;
+        t += (uint64_t)m[2] * v.z;
+        t += (uint64_t)m[3] * v.w;
+        h = t;
+    }
 }
 
 // Per-lane state of one tile's scan: the lane's four slot multipliers, its share
 // of the hash recurrence, and its fp64 accumulators.  Rows may be fed from
 // registers (direct loads) or from shared memory (bulk-async ring); the
 // arithmetic is the same.
-template <int DT>
+template <int DT, bool PTX_CHAIN = false>
 struct TileScan {
     uint32_t m[4];
     uint64_t h;
@@ -281,10 +305,10 @@ struct TileScan {
         a = Acc{0.0, 0.0, 0.0, 0.0};
     }
     // the two halves of a row's work, separately (the cost microbenchmark times each alone)
-    __device__ __forceinline__ void row_hash(const uint4 &v) { fold_row(h, v, m); }
+    __device__ __forceinline__ void row_hash(const uint4 &v) { fold_row<PTX_CHAIN>(h, v, m); }
     __device__ __forceinline__ void row_stats(const uint4 &v) { stats_fast<DT>(v, a); }
     __device__ __forceinline__ void row(const uint4 &v) {
-        fold_row(h, v, m);
+        fold_row<PTX_CHAIN>(h, v, m);
         stats_fast<DT>(v, a);
     }
     // Warp reduction of what the lanes hold: hash share, sums, and whether any lane
@@ -331,10 +355,10 @@ struct TileScan {
 
 // Front end 0: one warp scans one tile with direct 16-byte loads, UNROLL rows in
 // flight, no overlap of a warp's own loads with its own arithmetic.
-template <int DT>
+template <int DT, bool PTX_CHAIN = false>
 __device__ __forceinline__ void scan_tile(const uint8_t *tile, uint32_t nbytes, uint32_t lane,
                                           TileRec &out) {
-    TileScan<DT> st;
+    TileScan<DT, PTX_CHAIN> st;
     st.begin(lane);
     const uint32_t full = nbytes / ROW_BYTES;
     const uint8_t *p = tile + 16u * lane;

@@ -83,7 +83,7 @@ __global__ void __launch_bounds__(SIGN_THREADS, PREFETCH ? SCOUT_MINBLOCKS_PF : 
         TileRec rec;
         if constexpr (DTSEL >= 0) {
             if (PREFETCH) scan_tile_prefetch<DTSEL>(tile, td.nbytes, lane, rec);
-            else          scan_tile<DTSEL>(tile, td.nbytes, lane, rec);
+            else          scan_tile<DTSEL, true>(tile, td.nbytes, lane, rec);
         } else {
             if (PREFETCH) scan_dispatch_prefetch(td.dtype, tile, td.nbytes, lane, rec);
             else          scan_dispatch(td.dtype, tile, td.nbytes, lane, rec);
@@ -95,7 +95,7 @@ __global__ void __launch_bounds__(SIGN_THREADS, PREFETCH ? SCOUT_MINBLOCKS_PF : 
 
 using SignKernel = void (*)(const SignArgs);
 // The direct-scan kernel for a front end (0 direct, 1 register prefetch) and a launch
-// whose tiles all have dtype `uniform` (specialised for fp32 and bf16), or mixed (-1).
+// whose tiles all have dtype `uniform` (specialised for fp32, bf16 and fp16), or mixed (-1).
 SignKernel direct_kernel(int prefetch, int uniform) {
     if (prefetch) {
         if (uniform == SCOUT_DT_F32) return sign_tiles_direct<1, SCOUT_DT_F32>;
@@ -104,6 +104,7 @@ SignKernel direct_kernel(int prefetch, int uniform) {
     }
     if (uniform == SCOUT_DT_F32) return sign_tiles_direct<0, SCOUT_DT_F32>;
     if (uniform == SCOUT_DT_BF16) return sign_tiles_direct<0, SCOUT_DT_BF16>;
+    if (uniform == SCOUT_DT_F16) return sign_tiles_direct<0, SCOUT_DT_F16>;
     return sign_tiles_direct<0, -1>;
 }
 

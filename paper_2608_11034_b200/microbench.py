@@ -26,7 +26,8 @@ def build() -> list:
     for name in ("pipe_rates", "row_cost"):
         exe = os.path.join(OUT, name)
         src = os.path.join(SRC, name + ".cu")
-        if not os.path.exists(exe) or os.path.getmtime(exe) < os.path.getmtime(src):
+        deps = [src] + [os.path.join(HERE, "csrc", h) for h in ("scout_scan.cuh", "scout_internal.h")]
+        if not os.path.exists(exe) or os.path.getmtime(exe) < max(os.path.getmtime(d) for d in deps):
             subprocess.check_call([os.environ.get("NVCC", "nvcc")] + FLAGS + ["-o", exe, src])
         exes.append(exe)
     return exes
