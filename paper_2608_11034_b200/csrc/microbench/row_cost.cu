@@ -34,8 +34,11 @@ __global__ void __launch_bounds__(256, 4) rows(const uint4 *in, TileRec *out, in
 #pragma unroll 1
     for (int it = 0; it < iters; ++it) {
         uint4 v[8];
+        // the address changes with the iteration, so that neither the loads nor anything computed
+        // from the loaded words alone can be moved out of the loop
+        const uint32_t b = base ^ ((uint32_t)(it & 1) << 4);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) v[u] = lds16(base + u * 512);
+        for (int u = 0; u < 8; ++u) v[u] = lds16(b + u * 512);
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             if (MODE == 0) st.row(v[u]);
