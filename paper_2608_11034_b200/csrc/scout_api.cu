@@ -365,7 +365,7 @@ int sign_all(scout_plan *p, cudaStream_t stream, scout_sig_t *d_sigs, CertifyOut
         p->timed_launches += 1;
     }
     rc = launch_finalize(p->d_chunks, p->chunks.size(), p->R, p->d_recs, p->tiles.size(),
-                         p->tile_bytes / ROW_BYTES, d_sigs, zero_out, stream);
+                         p->tile_bytes / ROW_BYTES, p->max_chunk_tiles, d_sigs, zero_out, stream);
     if (rc) return rc;
     return mark_launched(p, stream);
 }
@@ -837,7 +837,7 @@ int scout_certify_host(scout_plan_t *p, const void *const *h_ptrs, scout_report_
         }
     }
     rc = launch_finalize(p->d_chunks, p->chunks.size(), p->R, p->d_recs, NT, p->tile_bytes / ROW_BYTES,
-                         p->d_sigs, p->d_out, p->s_comp);
+                         p->max_chunk_tiles, p->d_sigs, p->d_out, p->s_comp);
     if (rc) return rc;
     if ((rc = mark_launched(p, p->s_comp))) return rc;
     return vote_and_report(p, p->s_comp, report, h_outliers, outlier_cap, h_undecided, undecided_cap);

@@ -222,8 +222,8 @@ int launch_bounded_wait_selftest(uint64_t limit_ns, uint64_t *d_out, cudaStream_
 
 // zero_out (may be null): a CertifyOut the finalise kernel clears for the vote that follows
 int launch_finalize(const ChunkDesc *chunks, uint64_t C, uint32_t R, const TileRec *recs,
-                    uint64_t tiles_per_replica, uint32_t tile_rows, scout_sig_t *d_sigs,
-                    CertifyOut *zero_out, cudaStream_t stream);
+                    uint64_t tiles_per_replica, uint32_t tile_rows, uint32_t max_chunk_tiles,
+                    scout_sig_t *d_sigs, CertifyOut *zero_out, cudaStream_t stream);
 
 int launch_vote(uint32_t R, uint64_t C, const scout_sig_t *d_sigs, uint8_t *d_status,
                 uint64_t *d_bitmap, scout_outlier_t *d_outliers, uint64_t outlier_cap,

@@ -627,7 +627,8 @@ __global__ void __launch_bounds__(FIN_THREADS) finalize_chunks(const ChunkDesc *
                                                                uint32_t R, const TileRec *recs,
                                                                uint64_t tiles_per_replica,
                                                                uint32_t tile_rows, uint64_t p_stride,
-                                                               scout_sig_t *sigs, CertifyOut *zero_out) {
+                                                               scout_sig_t *sigs, CertifyOut *zero_out,
+                                                               uint32_t rep_batch) {
     pdl_launch_dependents();
     pdl_wait();
     if (zero_out && blockIdx.x == 0 && threadIdx.x < sizeof(CertifyOut) / sizeof(uint64_t))
@@ -635,19 +636,21 @@ __global__ void __launch_bounds__(FIN_THREADS) finalize_chunks(const ChunkDesc *
     const uint32_t lane = threadIdx.x & 31u;
     const uint64_t warp = (uint64_t)blockIdx.x * (FIN_THREADS / 32) + (threadIdx.x >> 5);
     const uint64_t n_warps = (uint64_t)gridDim.x * (FIN_THREADS / 32);
-    // One item = one chunk and up to COMBINE_BATCH replicas of it: the chunk's geometry (its
-    // descriptor, the lanes' weights) is worked out once for them, and for chunks of at most
-    // 32 tiles their record loads are in flight together (a warp's items are a chain of
-    // dependent memory round trips, so fewer and wider items are what shortens the kernel).
-    const uint32_t groups = (R + COMBINE_BATCH - 1) / COMBINE_BATCH;
+    // One item = one chunk and up to rep_batch replicas of it (COMBINE_BATCH when no chunk of the
+    // plan has more than 32 tiles, else 1): the chunk's geometry (its descriptor, the lanes'
+    // weights) is worked out once for them and their record loads are in flight together.  A
+    // warp's items are a chain of dependent memory round trips, so for chunks of few tiles fewer
+    // and wider items shorten the kernel (24,320 chunks x 16 replicas: 231 -> 109 us); chunks of
+    // many tiles keep one item per replica (717 chunks of 512 tiles x 3: 13 us, 21 us if grouped).
+    const uint32_t groups = (R + rep_batch - 1) / rep_batch;
     for (uint64_t item = warp; item < C * groups; item += n_warps) {
         const uint64_t c = item / groups;
-        const uint32_t r0 = (uint32_t)(item - c * groups) * COMBINE_BATCH;
-        const uint32_t n_rep = min((uint32_t)COMBINE_BATCH, R - r0);
+        const uint32_t r0 = (uint32_t)(item - c * groups) * rep_batch;
+        const uint32_t n_rep = min(rep_batch, R - r0);
         const ChunkDesc cd = chunks[c];
         const uint64_t weight = combine_weight(cd.ntiles, cd.nbytes, tile_rows, lane);
         const TileRec *tr = recs + (uint64_t)r0 * tiles_per_replica + cd.tile0;
-        if (cd.ntiles <= 32u) {
+        if (rep_batch > 1) {   // every chunk of the plan has at most 32 tiles
             scout_sig_t o[COMBINE_BATCH];
             combine_small(tr, tiles_per_replica, n_rep, cd.ntiles, cd.nbytes, cd.k, cd.dtype, cd.meta, weight, lane, o);
 #pragma unroll
@@ -729,16 +732,17 @@ int launch_bounded_wait_selftest(uint64_t limit_ns, uint64_t *d_out, cudaStream_
 }
 
 int launch_finalize(const ChunkDesc *chunks, uint64_t C, uint32_t R, const TileRec *recs,
-                    uint64_t tiles_per_replica, uint32_t tile_rows, scout_sig_t *d_sigs,
-                    CertifyOut *zero_out, cudaStream_t stream) {
+                    uint64_t tiles_per_replica, uint32_t tile_rows, uint32_t max_chunk_tiles,
+                    scout_sig_t *d_sigs, CertifyOut *zero_out, cudaStream_t stream) {
     if (C == 0) return SCOUT_OK;
-    const uint64_t items = C * ((R + COMBINE_BATCH - 1) / COMBINE_BATCH);
+    const uint32_t rep_batch = max_chunk_tiles <= 32u ? (uint32_t)COMBINE_BATCH : 1u;
+    const uint64_t items = C * ((R + rep_batch - 1) / rep_batch);
     uint64_t blocks = (items + FIN_THREADS / 32 - 1) / (FIN_THREADS / 32);
     if (blocks > 148ull * 16) blocks = 148ull * 16;
     static_assert(sizeof(CertifyOut) / sizeof(uint64_t) <= FIN_THREADS, "one thread per word clears it");
     SCOUT_CUDA(launch_dependent(finalize_chunks, dim3((unsigned)blocks), dim3(FIN_THREADS), stream, chunks, C,
                                 R, recs, tiles_per_replica, tile_rows, pow_p(32ull * tile_rows), d_sigs,
-                                zero_out));
+                                zero_out, rep_batch));
     return SCOUT_OK;
 }
 
