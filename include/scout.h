@@ -270,15 +270,18 @@ SCOUT_API uint64_t scout_shape_tag(uint32_t ndim, const uint64_t *dims /*host*/)
 
 /* Knobs of a plan (optional).
  *   set "tile_bytes"  bytes per work item, a power of two in [2048, 262144]
- *   set "variant"     scan kernel: 0 = direct 16-byte loads (default); 1 = the same
- *                     with the next rows prefetched into registers; 2 = bulk-async
+ *   set "variant"     scan kernel: 1 (default) = 16-byte loads through a rotating
+ *                     register pipeline, eight rows always in flight, so that a warp's
+ *                     loads overlap its own arithmetic; 0 = the same loads in batches
+ *                     of eight rows without that overlap (the form the one-launch
+ *                     kernels use); 2 = bulk-async
  *                     copies (cp.async.bulk + mbarrier) through a per-warp ring in
  *                     shared memory; 4 = block-wide ring: a producer warp fetches
  *                     whole tiles (<= 32 KiB) with one bulk copy each and eight
  *                     consumer warps share them (needs tile_bytes <= 32768);
  *                     3 = read-only probe (measures the memory system only: the
  *                     records it leaves are NOT signatures)
- *   set "fused"       with the default scan (variant 0) and R <= 64 a call can run as
+ *   set "fused"       with the default scan (variants 0 and 1) and R <= 64 a call can run as
  *                     ONE kernel, in one of two forms.  1 = tickets: the warp that stores
  *                     the last tile record of a chunk finalises it (scout_sign_chunks), and
  *                     for scout_certify also votes it and folds it into the certificate

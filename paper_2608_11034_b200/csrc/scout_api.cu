@@ -48,7 +48,7 @@ struct scout_plan {
     std::vector<uint64_t> tensor_poff;    // [T+1] packed offsets, 256-byte aligned
     std::vector<TileDesc> tiles;
     uint32_t tile_bytes = 0;
-    int variant = 0, device = 0, grid = 0;
+    int variant = 1, device = 0, grid = 0;   // front end of the scan (key "variant"); 1 = register prefetch
     int uniform_dtype = -1;  // dtype of every tensor, or -1 if they differ
     bool bound = false;
 
@@ -71,7 +71,7 @@ struct scout_plan {
 
     // one-launch path (certify_tiles): per-chunk tickets, launch stamps, chain state
     int fused = -1;               // key "fused": 1 always, 0 never, -1 where it is the faster form (see
-                                  // launch_form); only the default scan (variant 0) has a one-launch form
+                                  // launch_form); the bulk-async front ends (variants 2, 4) have no one-launch form
     uint64_t total_bytes = 0;     // R * bytes per replica
     int fused_grid = 0;
     int cluster_ok = 0;           // the cluster form of the one-launch path can run this plan (upload_tables)
@@ -265,7 +265,7 @@ int upload_tables(scout_plan *p) {
 //     reaches 7.2 TB/s on 36 GB of fp32 and 6.5 TB/s on 125 GB of bf16; the ticket kernel
 //     stays 3 to 9 % below that, more than the three small launches it saves.
 int launch_form(const scout_plan *p, bool certify) {
-    if (p->variant != 0 || p->R > 64 || !p->d_tickets || p->fused == 0) return 0;
+    if (p->variant > 1 || p->R > 64 || !p->d_tickets || p->fused == 0) return 0;
     if (p->fused == 2) return p->cluster_ok ? 2 : 1;
     if (p->fused == 1) return 1;
     if (!certify || p->total_bytes >= (1ull << 30)) return 0;

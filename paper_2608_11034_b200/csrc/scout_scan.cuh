@@ -35,6 +35,7 @@ constexpr int SIGN_THREADS = 256;
 //   SCOUT_UNROLL         rows (16 B per lane each) a warp has in flight, direct scan
 //   SCOUT_MINBLOCKS      CTAs per SM the direct scan is compiled for (caps registers)
 //   SCOUT_MINBLOCKS_PF   the same for the register-prefetch front end
+//   SCOUT_PF_ROWS        rows the register-prefetch front end keeps in flight
 //   SCOUT_BF16_BITROUTE  see below
 //   SCOUT_RING_PIECE / _STAGES / _BLOCKS   geometry of the per-warp bulk-async ring
 #ifndef SCOUT_MINBLOCKS
@@ -375,18 +376,22 @@ __device__ __forceinline__ void scan_tile(const uint8_t *tile, uint32_t nbytes, 
     st.finish(tile, nbytes, lane, out);
 }
 
-// Front end 1: rotating register pipeline.  PF_ROWS rows are always in flight:
-// as soon as a row has been folded its registers are reloaded with the row
-// PF_ROWS ahead, so a warp's loads overlap its own arithmetic.
+// Front end 1 (the default of the staged scan): rotating register pipeline.  PF_ROWS rows
+// are always in flight: as soon as a row has been folded its registers are reloaded with
+// the row PF_ROWS ahead, so a warp's loads overlap its own arithmetic.  80 registers, three
+// CTAs per SM.  Measured against front end 0 in one session (GB/s, whole step): 36 GB of
+// fp32 7,039-7,063 -> 7,226-7,236 (the scan kernel at 0.99 of the read probe), 125 GB of bf16
+// 6,511-6,521 -> 6,554-6,577, 71 GB of mixed tensors 7,010 -> 7,120-7,143; depths 6, 10, 12
+// and 16 rows and 64 or 128 registers were equal or slower.
 #ifndef SCOUT_PF_ROWS
-#define SCOUT_PF_ROWS 4
+#define SCOUT_PF_ROWS 8
 #endif
 constexpr int PF_ROWS = SCOUT_PF_ROWS;
 
-template <int DT>
+template <int DT, bool PTX_CHAIN = false>
 __device__ __forceinline__ void scan_tile_prefetch(const uint8_t *tile, uint32_t nbytes, uint32_t lane,
                                                    TileRec &out) {
-    TileScan<DT> st;
+    TileScan<DT, PTX_CHAIN> st;
     st.begin(lane);
     const uint32_t full = nbytes / ROW_BYTES;
     const uint8_t *p = tile + 16u * lane;

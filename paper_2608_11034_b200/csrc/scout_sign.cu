@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(SIGN_THREADS, PREFETCH ? SCOUT_MINBLOCKS_PF : 
         const uint8_t *tile = tile_address(a, td, r);
         TileRec rec;
         if constexpr (DTSEL >= 0) {
-            if (PREFETCH) scan_tile_prefetch<DTSEL>(tile, td.nbytes, lane, rec);
+            if (PREFETCH) scan_tile_prefetch<DTSEL, true>(tile, td.nbytes, lane, rec);
             else          scan_tile<DTSEL, true>(tile, td.nbytes, lane, rec);
         } else {
             if (PREFETCH) scan_dispatch_prefetch(td.dtype, tile, td.nbytes, lane, rec);

@@ -69,7 +69,7 @@ def gpu_plan(w, chunk_bytes=None, tags=None, tile_bytes=None, variant=None):
                         w.chunk_bytes if chunk_bytes is None else chunk_bytes, guards=True)
     if tile_bytes is not None:
         binding.scout_plan_set(plan.handle, "tile_bytes", tile_bytes)
-    if variant == "unfused":      # the default scan, one kernel per stage
+    if variant == "unfused":      # the default scan (register-prefetch front end), one kernel per stage
         binding.scout_plan_set(plan.handle, "fused", 0)
     elif variant == "fused":      # the default scan, the whole call as one launch (tickets)
         binding.scout_plan_set(plan.handle, "fused", 1)

@@ -18,7 +18,7 @@ def test_plan_knobs():
     plan = helpers.gpu_plan(w)
     h = plan.handle
     assert B.scout_plan_get(h, "tile_bytes") in (4096, 8192, 16384, 32768)
-    assert B.scout_plan_get(h, "variant") == 0 and B.scout_plan_get(h, "grid") > 0
+    assert B.scout_plan_get(h, "variant") == 1 and B.scout_plan_get(h, "grid") > 0
     n0 = B.scout_plan_get(h, "n_tiles")
     B.scout_plan_set(h, "tile_bytes", 2048)
     assert B.scout_plan_get(h, "n_tiles") == w.bytes_per_replica // 2048 != n0

@@ -22,7 +22,7 @@ def _binding():
 
 # direct loads with one kernel per stage, the same scan with the whole call as one launch, register
 # prefetch, per-warp bulk-async ring, block-wide ring
-VARIANTS = ["unfused", "fused", "cluster", 1, 2, 4]
+VARIANTS = ["unfused", "fused", "cluster", 0, 1, 2, 4]   # "unfused": the default front end (1), one kernel per stage
 
 
 def _compare_everything(w, views, chunk_bytes=None, tile_bytes=None, variant=None):
@@ -69,7 +69,7 @@ def _odd_workload(dtype, seed):
 
 @pytest.mark.parametrize("dtype", ["u8", "f32", "bf16", "i64", "f16", "f64", "i32"])
 @pytest.mark.parametrize("tile_bytes,variant", [(2048, "fused"), (4096, "fused"), (2048, "cluster"), (4096, "cluster"), (2048, "unfused"), (4096, "unfused"),
-                                                (4096, 1), (8192, 1),
+                                                (4096, 0), (8192, 0), (4096, 1), (8192, 1),
                                                 (4096, 2), (8192, 2), (32768, 2), (4096, 4), (8192, 4), (32768, 4)])
 def test_every_dtype_and_ragged_sizes(dtype, tile_bytes, variant):
     w = _odd_workload(dtype, 77)
@@ -211,7 +211,7 @@ def test_results_are_bitwise_reproducible_and_independent_of_tiling():
     a = helpers.gpu_sign_vote(w, views)
     b = helpers.gpu_sign_vote(w, views)
     assert a["sigs"].tobytes() == b["sigs"].tobytes()
-    for tile, variant in ((2048, "fused"), (32768, "fused"), (2048, "unfused"), (32768, "unfused"), (8192, 1), (32768, 2), (65536, 2), (65536, 1), (32768, 4), (2048, 4)):
+    for tile, variant in ((2048, "fused"), (32768, "fused"), (2048, "unfused"), (32768, "unfused"), (8192, 0), (32768, 0), (8192, 1), (32768, 2), (65536, 2), (65536, 1), (32768, 4), (2048, 4)):
         c = helpers.gpu_sign_vote(w, views, tile_bytes=tile, variant=variant)
         assert (c["sigs"]["hash"] == a["sigs"]["hash"]).all()
         assert c["outliers"] == a["outliers"]
