@@ -258,11 +258,14 @@ __device__ __noinline__ void rescan_classifying(const uint8_t *tile, uint32_t nb
 // arithmetic.  From the C++ expression the compiler makes 11 instructions per row; from
 // the PTX chain the 7 it needs (one wide multiply and two 32-bit multiply-adds for h * P,
 // four wide multiply-adds).  Which one is faster depends on what surrounds it (measured
-// in one session, 3 GB to 125 GB per step): in the kernels compiled for a single element
-// type the PTX chain wins (fp32 6,905-6,918 -> 7,027-7,034 GB/s, bf16 6,352-6,381 ->
-// 6,470-6,490), in the kernel that reads the type from the tile table the C++ form does
-// (int64 7,198 against 7,009, uint8 7,194 / 6,990, int32 7,175 / 6,799, fp64 6,883 /
-// 6,803; mixed fp32/bf16/int64 equal).  So PTX_CHAIN is set by the single-type kernels only.
+// in one session, 3 GB to 125 GB per step).  In the kernels compiled for a single element
+// type the PTX chain wins (front end 0: fp32 6,905-6,918 -> 7,027-7,034 GB/s, bf16
+// 6,352-6,381 -> 6,470-6,490).  In the kernel that reads the type from the tile table it
+// depends on the front end: with batches of rows (front end 0) the C++ form wins (int64
+// 7,198 against 7,009, uint8 7,194 / 6,990, int32 7,175 / 6,799, fp64 6,883 / 6,803), with
+// the register pipeline (front end 1) the PTX chain does (10,000 mixed tensors 7,124 ->
+// 7,167-7,178, int32 6,921 -> 6,955, the others equal).  Each kernel uses what measured
+// faster for it.
 template <bool PTX_CHAIN>
 __device__ __forceinline__ void fold_row(uint64_t &h, const uint4 &v, const uint32_t (&m)[4]) {
     if constexpr (PTX_CHAIN) {
@@ -387,6 +390,8 @@ __device__ __forceinline__ void scan_tile(const uint8_t *tile, uint32_t nbytes, 
 #define SCOUT_PF_ROWS 8
 #endif
 constexpr int PF_ROWS = SCOUT_PF_ROWS;
+// spelling of the hash fold in the mixed-type kernel of this front end (see fold_row)
+constexpr bool MIXED_PTX_CHAIN = true;
 
 template <int DT, bool PTX_CHAIN = false>
 __device__ __forceinline__ void scan_tile_prefetch(const uint8_t *tile, uint32_t nbytes, uint32_t lane,
@@ -452,13 +457,13 @@ __device__ __forceinline__ void scan_dispatch(uint32_t dtype, const uint8_t *til
 __device__ __forceinline__ void scan_dispatch_prefetch(uint32_t dtype, const uint8_t *tile,
                                                        uint32_t nbytes, uint32_t lane, TileRec &rec) {
     switch (dtype) {
-        case SCOUT_DT_F32:  scan_tile_prefetch<SCOUT_DT_F32>(tile, nbytes, lane, rec); break;
-        case SCOUT_DT_BF16: scan_tile_prefetch<SCOUT_DT_BF16>(tile, nbytes, lane, rec); break;
-        case SCOUT_DT_I64:  scan_tile_prefetch<SCOUT_DT_I64>(tile, nbytes, lane, rec); break;
-        case SCOUT_DT_F16:  scan_tile_prefetch<SCOUT_DT_F16>(tile, nbytes, lane, rec); break;
-        case SCOUT_DT_F64:  scan_tile_prefetch<SCOUT_DT_F64>(tile, nbytes, lane, rec); break;
-        case SCOUT_DT_I32:  scan_tile_prefetch<SCOUT_DT_I32>(tile, nbytes, lane, rec); break;
-        default:            scan_tile_prefetch<SCOUT_DT_U8>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_F32:  scan_tile_prefetch<SCOUT_DT_F32, MIXED_PTX_CHAIN>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_BF16: scan_tile_prefetch<SCOUT_DT_BF16, MIXED_PTX_CHAIN>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_I64:  scan_tile_prefetch<SCOUT_DT_I64, MIXED_PTX_CHAIN>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_F16:  scan_tile_prefetch<SCOUT_DT_F16, MIXED_PTX_CHAIN>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_F64:  scan_tile_prefetch<SCOUT_DT_F64, MIXED_PTX_CHAIN>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_I32:  scan_tile_prefetch<SCOUT_DT_I32, MIXED_PTX_CHAIN>(tile, nbytes, lane, rec); break;
+        default:            scan_tile_prefetch<SCOUT_DT_U8, MIXED_PTX_CHAIN>(tile, nbytes, lane, rec); break;
     }
 }
 
