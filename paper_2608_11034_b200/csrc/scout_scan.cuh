@@ -51,10 +51,11 @@ constexpr int SIGN_THREADS = 256;
 
 constexpr int UNROLL = SCOUT_UNROLL;
 // bf16: how many of a word-quad's four high halves are widened by bit placement
-// instead of the conversion pipe (see stats_fast).  Default 0: every instruction costs about
-// 1.6 issue cycles whatever its pipe, so the route with the fewest instructions wins even
-// though it keeps the conversion pipe busiest (measured on 125 GB of bf16: 6,361 GB/s with 0,
-// 6,282 with 1, 6,223 with 2, 6,016 with 3).
+// instead of the conversion pipe (see stats_fast), in every front end but the register
+// pipeline (which has its own setting, PF_BITROUTE).  Default 0: where a warp also sits out
+// its own load latency every instruction costs about 1.6 issue cycles whatever its pipe, so
+// the route with the fewest instructions wins even though it keeps the conversion pipe
+// busiest (measured on 125 GB of bf16: 6,361 GB/s with 0, 6,282 with 1, 6,223 with 2, 6,016 with 3).
 #ifndef SCOUT_BF16_BITROUTE
 #define SCOUT_BF16_BITROUTE 0
 #endif
@@ -98,7 +99,7 @@ __device__ __forceinline__ void acc2(Acc &a, double x0, double x1) {
 }
 
 // ---- per-dtype element paths: fast (no classification) -----------------------
-template <int DT>
+template <int DT, int BITROUTE = BF16_BITROUTE>
 __device__ __forceinline__ void stats_fast(const uint4 &v, Acc &a) {
     if constexpr (DT == SCOUT_DT_F32) {
         acc2(a, (double)__uint_as_float(v.x), (double)__uint_as_float(v.y));
@@ -127,7 +128,7 @@ __device__ __forceinline__ void stats_fast(const uint4 &v, Acc &a) {
             asm("cvt.f64.bf16 %0, %1;" : "=d"(lo) : "h"(l16));
             a.s0 += lo;
             a.q0 = fma(lo, lo, a.q0);
-            if (i < BF16_BITROUTE) {
+            if (i < BITROUTE) {
                 const uint32_t uh = (uint32_t)((int)w[i] >> 3) & 0x8FFFE000u;
                 const double u = __hiloint2double((int)uh, 0);
                 const double x2 = __hiloint2double((int)(uh | 0x70000000u), 0);
@@ -136,7 +137,7 @@ __device__ __forceinline__ void stats_fast(const uint4 &v, Acc &a) {
             } else {
                 double hi;
                 asm("cvt.f64.bf16 %0, %1;" : "=d"(hi) : "h"(h16));
-                if (BF16_BITROUTE > 0) {
+                if (BITROUTE > 0) {
                     a.s0 += hi;
                     a.q0 = fma(hi, hi, a.q0);
                 } else {
@@ -167,12 +168,12 @@ __device__ __forceinline__ void stats_fast(const uint4 &v, Acc &a) {
     }
 }
 
-template <int DT>
+template <int DT, int BITROUTE = BF16_BITROUTE>
 __device__ __forceinline__ bool may_hold_nonfinite(const Acc &a) {
     if constexpr (DT == SCOUT_DT_BF16) {
         // non-finite element, or a subnormal one on the bit-placement route
         return !(a.q0 + a.q1 < 1.157920892373162e77) ||                    // 2^256
-               (BF16_BITROUTE > 0 && a.q1 > 0.0 && a.q1 < 6.525304467998525e-55);  // 2^-180
+               (BITROUTE > 0 && a.q1 > 0.0 && a.q1 < 6.525304467998525e-55);  // 2^-180
     } else if constexpr (DT == SCOUT_DT_F32 || DT == SCOUT_DT_F16) {
         return !(a.q0 + a.q1 < 1.157920892373162e77);  // 2^256
     } else if constexpr (DT == SCOUT_DT_F64) {
@@ -296,7 +297,7 @@ __device__ __forceinline__ void fold_row(uint64_t &h, const uint4 &v, const uint
 // of the hash recurrence, and its fp64 accumulators.  Rows may be fed from
 // registers (direct loads) or from shared memory (bulk-async ring); the
 // arithmetic is the same.
-template <int DT, bool PTX_CHAIN = false>
+template <int DT, bool PTX_CHAIN = false, int BITROUTE = BF16_BITROUTE>
 struct TileScan {
     uint32_t m[4];
     uint64_t h;
@@ -310,20 +311,20 @@ struct TileScan {
     }
     // the two halves of a row's work, separately (the cost microbenchmark times each alone)
     __device__ __forceinline__ void row_hash(const uint4 &v) { fold_row<PTX_CHAIN>(h, v, m); }
-    __device__ __forceinline__ void row_stats(const uint4 &v) { stats_fast<DT>(v, a); }
+    __device__ __forceinline__ void row_stats(const uint4 &v) { stats_fast<DT, BITROUTE>(v, a); }
     __device__ __forceinline__ void row(const uint4 &v) {
         fold_row<PTX_CHAIN>(h, v, m);
-        stats_fast<DT>(v, a);
+        stats_fast<DT, BITROUTE>(v, a);
     }
     // Warp reduction of what the lanes hold: hash share, sums, and whether any lane
     // suspects a non-finite (or, for bf16, subnormal) element.
     __device__ __forceinline__ void reduce(uint64_t &h_out, double &s, double &q, bool &suspect) const {
         q = a.q0 + a.q1;
-        if constexpr (DT == SCOUT_DT_BF16 && BF16_BITROUTE > 0)
+        if constexpr (DT == SCOUT_DT_BF16 && BITROUTE > 0)
             s = fma(a.s1, 0x1p896, a.s0);  // s1 holds x * 2^-896: exact power-of-two rescale
         else
             s = a.s0 + a.s1;
-        suspect = __any_sync(0xFFFFFFFFu, may_hold_nonfinite<DT>(a));
+        suspect = __any_sync(0xFFFFFFFFu, may_hold_nonfinite<DT, BITROUTE>(a));
         h_out = h;
 #pragma unroll
         for (int d = 16; d >= 1; d >>= 1) {
@@ -392,11 +393,20 @@ __device__ __forceinline__ void scan_tile(const uint8_t *tile, uint32_t nbytes, 
 constexpr int PF_ROWS = SCOUT_PF_ROWS;
 // spelling of the hash fold in the mixed-type kernel of this front end (see fold_row)
 constexpr bool MIXED_PTX_CHAIN = true;
+// bf16 elements per word quad that this front end widens by bit placement (see stats_fast).
+// With the loads overlapped the conversion pipe is the busiest unit of the bf16 scan (75 %),
+// and unloading a quarter of its work for six more instructions per row pays: 125 GB of bf16
+// 6,558 (none) / 6,548 (one) / 6,654-6,681 (two) / 6,645 (three).  Front end 0, whose warps
+// also have their own load latency to sit out, is fastest with none (6,361 / 6,282 / 6,223 / 6,016).
+constexpr int PF_BITROUTE = 2;
+// ... and in the mixed-type kernel of this front end, where none is faster (10,000 mixed
+// tensors: 7,172-7,176 with none, 7,118-7,137 with two)
+constexpr int MIXED_PF_BITROUTE = 0;
 
-template <int DT, bool PTX_CHAIN = false>
+template <int DT, bool PTX_CHAIN = false, int BITROUTE = PF_BITROUTE>
 __device__ __forceinline__ void scan_tile_prefetch(const uint8_t *tile, uint32_t nbytes, uint32_t lane,
                                                    TileRec &out) {
-    TileScan<DT, PTX_CHAIN> st;
+    TileScan<DT, PTX_CHAIN, BITROUTE> st;
     st.begin(lane);
     const uint32_t full = nbytes / ROW_BYTES;
     const uint8_t *p = tile + 16u * lane;
@@ -457,13 +467,13 @@ __device__ __forceinline__ void scan_dispatch(uint32_t dtype, const uint8_t *til
 __device__ __forceinline__ void scan_dispatch_prefetch(uint32_t dtype, const uint8_t *tile,
                                                        uint32_t nbytes, uint32_t lane, TileRec &rec) {
     switch (dtype) {
-        case SCOUT_DT_F32:  scan_tile_prefetch<SCOUT_DT_F32, MIXED_PTX_CHAIN>(tile, nbytes, lane, rec); break;
-        case SCOUT_DT_BF16: scan_tile_prefetch<SCOUT_DT_BF16, MIXED_PTX_CHAIN>(tile, nbytes, lane, rec); break;
-        case SCOUT_DT_I64:  scan_tile_prefetch<SCOUT_DT_I64, MIXED_PTX_CHAIN>(tile, nbytes, lane, rec); break;
-        case SCOUT_DT_F16:  scan_tile_prefetch<SCOUT_DT_F16, MIXED_PTX_CHAIN>(tile, nbytes, lane, rec); break;
-        case SCOUT_DT_F64:  scan_tile_prefetch<SCOUT_DT_F64, MIXED_PTX_CHAIN>(tile, nbytes, lane, rec); break;
-        case SCOUT_DT_I32:  scan_tile_prefetch<SCOUT_DT_I32, MIXED_PTX_CHAIN>(tile, nbytes, lane, rec); break;
-        default:            scan_tile_prefetch<SCOUT_DT_U8, MIXED_PTX_CHAIN>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_F32:  scan_tile_prefetch<SCOUT_DT_F32, MIXED_PTX_CHAIN, MIXED_PF_BITROUTE>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_BF16: scan_tile_prefetch<SCOUT_DT_BF16, MIXED_PTX_CHAIN, MIXED_PF_BITROUTE>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_I64:  scan_tile_prefetch<SCOUT_DT_I64, MIXED_PTX_CHAIN, MIXED_PF_BITROUTE>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_F16:  scan_tile_prefetch<SCOUT_DT_F16, MIXED_PTX_CHAIN, MIXED_PF_BITROUTE>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_F64:  scan_tile_prefetch<SCOUT_DT_F64, MIXED_PTX_CHAIN, MIXED_PF_BITROUTE>(tile, nbytes, lane, rec); break;
+        case SCOUT_DT_I32:  scan_tile_prefetch<SCOUT_DT_I32, MIXED_PTX_CHAIN, MIXED_PF_BITROUTE>(tile, nbytes, lane, rec); break;
+        default:            scan_tile_prefetch<SCOUT_DT_U8, MIXED_PTX_CHAIN, MIXED_PF_BITROUTE>(tile, nbytes, lane, rec); break;
     }
 }
 
