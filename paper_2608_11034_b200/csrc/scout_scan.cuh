@@ -36,6 +36,7 @@ constexpr int SIGN_THREADS = 256;
 //   SCOUT_MINBLOCKS      CTAs per SM the direct scan is compiled for (caps registers)
 //   SCOUT_MINBLOCKS_PF   the same for the register-prefetch front end
 //   SCOUT_PF_ROWS        rows the register-prefetch front end keeps in flight
+//   SCOUT_PF_BITROUTE    bf16 elements per word quad it widens by bit placement
 //   SCOUT_BF16_BITROUTE  see below
 //   SCOUT_RING_PIECE / _STAGES / _BLOCKS   geometry of the per-warp bulk-async ring
 #ifndef SCOUT_MINBLOCKS
@@ -398,7 +399,10 @@ constexpr bool MIXED_PTX_CHAIN = true;
 // and unloading a quarter of its work for six more instructions per row pays: 125 GB of bf16
 // 6,558 (none) / 6,548 (one) / 6,654-6,681 (two) / 6,645 (three).  Front end 0, whose warps
 // also have their own load latency to sit out, is fastest with none (6,361 / 6,282 / 6,223 / 6,016).
-constexpr int PF_BITROUTE = 2;
+#ifndef SCOUT_PF_BITROUTE
+#define SCOUT_PF_BITROUTE 2
+#endif
+constexpr int PF_BITROUTE = SCOUT_PF_BITROUTE;
 // ... and in the mixed-type kernel of this front end, where none is faster (10,000 mixed
 // tensors: 7,172-7,176 with none, 7,118-7,137 with two)
 constexpr int MIXED_PF_BITROUTE = 0;
