@@ -50,7 +50,7 @@ SCAN_TRAFFIC_SOURCE = ("ncu capture of the scan kernel on 1.8 GB at commit a9c02
 # SM cycles per 512-byte row and scheduler of the scan's row routine with its data already on the
 # SM (`python -m paper_2608_11034_b200.microbench`, its output is summarised under profiles/): the
 # compute bound of a uniform-dtype workload at SM clock f is 512 B * 4 * SMs * f / cycles.
-ROW_COST_CYCLES = {"bf16": 75.5, "f16": 75.6, "f32": 45.1, "i64": 41.2, "u8": 28.1}
+ROW_COST_CYCLES = {"bf16": 74.7, "f16": 75.6, "f32": 45.1, "i64": 41.2, "u8": 28.1}
 N_SMS = 148
 
 

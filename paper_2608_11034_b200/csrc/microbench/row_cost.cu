@@ -21,7 +21,7 @@ static __device__ __forceinline__ uint4 lds16(uint32_t addr) {
     return v;
 }
 
-template <int DT, int MODE, bool PTX_CHAIN>
+template <int DT, int MODE, bool PTX_CHAIN, int BITROUTE = 0>
 __global__ void __launch_bounds__(256, 4) rows(const uint4 *in, TileRec *out, int iters) {
     extern __shared__ __align__(16) uint8_t sm[];
     const uint32_t lane = threadIdx.x & 31u, wib = threadIdx.x >> 5;
@@ -29,7 +29,7 @@ __global__ void __launch_bounds__(256, 4) rows(const uint4 *in, TileRec *out, in
     for (int u = 0; u < 8; ++u) mine[u * 32 + lane] = in[(blockIdx.x * 8 + wib) % 64 * 256 + u * 32 + lane];
     __syncthreads();
     const uint32_t base = smem_u32(mine) + 16u * lane;
-    TileScan<DT, PTX_CHAIN> st;
+    TileScan<DT, PTX_CHAIN, BITROUTE> st;
     st.begin(lane);
 #pragma unroll 1
     for (int it = 0; it < iters; ++it) {
@@ -54,25 +54,25 @@ __global__ void __launch_bounds__(256, 4) rows(const uint4 *in, TileRec *out, in
 static double g_mhz = 1965.0;
 static int g_sms = 148;
 
-template <int DT, int MODE, bool PTX_CHAIN>
+template <int DT, int MODE, bool PTX_CHAIN, int BITROUTE = 0>
 void run(const char *dtype, const uint4 *in, TileRec *out) {
     static const char *mode[3] = {"hash + statistics", "hash only", "statistics only"};
     const int iters = 2000;
-    cudaFuncSetAttribute(rows<DT, MODE, PTX_CHAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768);
+    cudaFuncSetAttribute(rows<DT, MODE, PTX_CHAIN, BITROUTE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768);
     for (int per_sm = 1; per_sm <= 4; per_sm *= 2) {
-        rows<DT, MODE, PTX_CHAIN><<<g_sms * per_sm, 256, 32768>>>(in, out, iters);
+        rows<DT, MODE, PTX_CHAIN, BITROUTE><<<g_sms * per_sm, 256, 32768>>>(in, out, iters);
         cudaDeviceSynchronize();
         cudaEvent_t e0, e1;
         cudaEventCreate(&e0); cudaEventCreate(&e1);
         cudaEventRecord(e0);
-        rows<DT, MODE, PTX_CHAIN><<<g_sms * per_sm, 256, 32768>>>(in, out, iters);
+        rows<DT, MODE, PTX_CHAIN, BITROUTE><<<g_sms * per_sm, 256, 32768>>>(in, out, iters);
         cudaEventRecord(e1);
         cudaDeviceSynchronize();
         float ms = 0.f;
         cudaEventElapsedTime(&ms, e0, e1);
         const double rows_per_sched = 2.0 * per_sm * iters * 8.0;
         const double cyc = ms * 1e-3 * g_mhz * 1e6 / rows_per_sched;
-        printf("%-16s %-18s %d warps/scheduler: %6.2f cycles per row per scheduler -> %6.0f GB/s at %.0f MHz\n", dtype,
+        printf("%-20s %-18s %d warps/scheduler: %6.2f cycles per row per scheduler -> %6.0f GB/s at %.0f MHz\n", dtype,
                mode[MODE], 2 * per_sm, cyc, 512.0 * 4 * g_sms * g_mhz * 1e6 / cyc / 1e9, g_mhz);
         cudaEventDestroy(e0); cudaEventDestroy(e1);
     }
@@ -97,6 +97,9 @@ int main(int argc, char **argv) {
     cudaMemcpy(in, h, 64 * 4096, cudaMemcpyHostToDevice);
     // the kernels compiled for one element type (fp32, bf16, fp16) use the PTX spelling of the hash
     // fold, the kernel that reads the type from the tile table the C++ one: see fold_row
+    // bf16 as the default kernel runs it: two of eight elements widened by bit placement
+    run<SCOUT_DT_BF16, 0, true, PF_BITROUTE>("bf16 (2 of 8 placed)", in, out);
+    run<SCOUT_DT_BF16, 2, true, PF_BITROUTE>("bf16 (2 of 8 placed)", in, out);
     run<SCOUT_DT_BF16, 0, true>("bf16", in, out); run<SCOUT_DT_BF16, 1, true>("bf16", in, out);
     run<SCOUT_DT_BF16, 2, true>("bf16", in, out);
     run<SCOUT_DT_F32, 0, true>("f32", in, out);   run<SCOUT_DT_F32, 2, true>("f32", in, out);
