@@ -689,7 +689,16 @@ def main():
     if also:
         line["also"] = {}
         for cfg in also:
-            r = run_config(cfg, args, rank, world, local, headline=False)
+            # a config that cannot run here (say, a board with less free memory) or that fails its own
+            # check is reported as such; it does not take the headline line down with it
+            try:
+                r = run_config(cfg, args, rank, world, local, headline=False)
+            except (Exception, SystemExit) as e:                       # noqa: BLE001
+                line["also"][f"cfg{cfg}"] = {"error": repr(e)[:300], "verified": False}
+                import gc
+                gc.collect()
+                torch.cuda.empty_cache()
+                continue
             line["also"][r["config"]["workload"]] = {
                 "value": r["value"], "ms_per_step": r["ms_per_step"],
                 "bytes_per_step": r["config"]["bytes_per_step_per_gpu"],
