@@ -214,3 +214,34 @@ def test_the_default_picks_the_form_by_shape():
     assert form(3, 1 << 20, 4 << 20) == (0, 0)          # one chunk of 1,024 tiles, 12.6 MB: per stage
     assert form(3, 16 << 20, 4 << 20) == (0, 0)         # 201 MB in 4 MiB chunks (256 tiles each): per stage
     assert form(3, 2 << 20, 2048) == (0, 0)             # 4,096 chunks: the chain decides, per stage
+
+
+def test_several_plans_in_flight_on_different_streams():
+    """Six plans of different shapes, each in the form the library picks for it (clusters,
+    tickets, one kernel per stage), launched on six streams before any is collected, 300 times
+    over: every report equals the plan's own staged result (no state is shared between plans,
+    and every launch leaves its plan's device state ready for the next)."""
+    from paper_2608_11034_b200 import binding as B
+    ws = [inputs.workload(1, "default", 1.0), inputs.workload(2, "mantissa", 0.25), inputs.workload(3, "default", 0.002),
+          inputs.workload(1, "default", 0.5), inputs.workload(5, "default", 0.005), inputs.workload(4, "default", 0.002)]
+    plans, refs, streams, keep = [], [], [], []
+    for w in ws:
+        _, views = inputs.generate(w, "cuda")
+        keep.append(views)
+        p = helpers.gpu_plan(w)
+        p.bind(views)
+        B.scout_plan_set(p.handle, "fused", 0)
+        refs.append(p.certify())
+        B.scout_plan_set(p.handle, "fused", -1)
+        plans.append(p)
+        streams.append(torch.cuda.Stream())
+    assert {B.scout_plan_get(p.handle, "certify_form") for p in plans} == {0, 1, 2}
+    for _ in range(300):
+        for p, s in zip(plans, streams):
+            p.certify_launch(stream=s.cuda_stream)
+        for p, ref in zip(plans, refs):
+            got = p.certify_collect()
+            assert got["report"] == ref["report"] and got["outliers"] == ref["outliers"]
+    for p in plans:
+        helpers.assert_guards(p)
+        p.close()
